@@ -1,0 +1,239 @@
+"""Plain fp64 CPU oracle for ST^3 decode-step attention over a trimmed visual KV cache.
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  It shares no code with the CUDA path and is not
+tuned for speed.  Every function restates a passage of the paper (ST^3,
+"Spatial-Temporal Visual Token Trimming") step by step in numpy float64.
+
+Readings taken where the paper is silent or inconsistent (each one is a
+documented choice, not a derivation):
+  * PVTP ratios are additive in the ORIGINAL visual-token count: the first
+    pruning layer removes P, each later pruning layer removes a further R.
+    This is the reading that reproduces every (L, S, R) -> C row the paper
+    prints in its stride/ratio ablation tables.
+  * Pruning layers are l = first, first+S, first+2S, ... (first = 3); the
+    layers between two pruning layers keep the count of their stage.
+  * VTA count is |V^{l,0}| * beta^t (Eq. 7, non-compounding), floor'ed; with
+    |O^t| = t at decode step t (t = 1 consumes the first generated token).
+  * The score of a visual token is the sum over heads of the current query's
+    attention probability on it (Eq. 2's last row, sliced to visual positions).
+  * Top(G, .) breaks equal scores toward the lower original visual index.
+  * Attend first, then trim: the cache after step t holds n(l, t) visual rows.
+  * Selection at layer l uses layer l's own scores (layer-local trimming).
+
+Pins (tests/test_oracle_*.py): the paper's printed (L, S, R, C) table rows,
+closed forms of beta, brute-force softmax in long double, torch SDPA as a
+library special case, an O(n^2) exhaustive definition of top-k, and run-long
+invariants.  No function here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass, field
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------
+# Retention schedule: PVTP per layer (Sec. 3.2, Eq. 9, Algorithm 1) times
+# VTA per decode step (Sec. 3.3, Eq. 7 and Eq. 8).
+# --------------------------------------------------------------------------
+@dataclass(frozen=True)
+class Schedule:
+    num_layers: int
+    num_visual: int
+    stride: int                      # S, pruning stride
+    step_ratio_bp: int               # R in basis points of num_visual
+    tau: float                       # Eq. 8 decay horizon
+    first_ratio_bp: int = 5000       # P, "set to 50%" (text under Eq. 9)
+    first_prune_layer: int = 3       # "avoid pruning tokens in the first three layers"
+    anneal: str = "cosine"           # "cosine" | "linear" | "exp" | "none"
+    sigma: float = 20.0              # only for anneal == "exp"
+    disable_trim: bool = False       # full-KV comparison run
+
+    def stage(self, layer: int) -> int:
+        """Index of the pruning stage layer `layer` belongs to (-1: never pruned).
+
+        Algorithm 1 prunes when l >= 3 and (l - 3) % S == 0, so stage heads are
+        3, 3+S, 3+2S, ... and every layer up to the next head shares the stage.
+        """
+        if layer < self.first_prune_layer:
+            return -1
+        return (layer - self.first_prune_layer) // self.stride
+
+    def keep_bp(self, layer: int) -> int:
+        """Fraction of the original visual tokens layer `layer` keeps, in basis points.
+
+        Eq. 9 generalised to every layer: 1 - P - k*R with k the number of
+        pruning layers passed after the first one.
+        """
+        k = self.stage(layer)
+        if k < 0 or self.disable_trim:
+            return 10000
+        return max(0, 10000 - self.first_ratio_bp - k * self.step_ratio_bp)
+
+    def n0(self, layer: int) -> int:
+        """|V^{l,0}|: visual tokens kept at layer l after prefill (floor)."""
+        return (self.num_visual * self.keep_bp(layer)) // 10000
+
+    def beta(self, t: int) -> float:
+        """Eq. 8 (cosine), or the linear / exponential variants of Sec. 4.4."""
+        if self.anneal == "none" or self.disable_trim:
+            return 1.0
+        if self.anneal == "exp":
+            return math.exp(-t / self.sigma)
+        if t >= self.tau:
+            return 0.0
+        if self.anneal == "cosine":
+            return math.cos(t * math.pi / (2.0 * self.tau))
+        if self.anneal == "linear":
+            return 1.0 - t / self.tau
+        raise ValueError(self.anneal)
+
+    def n(self, layer: int, t: int) -> int:
+        """Scheduled visual-row count of layer `layer` after decode step t (Eq. 7)."""
+        base = self.n0(layer)
+        if layer < self.first_prune_layer or t == 0:
+            return base
+        return int(math.floor(base * self.beta(t) + 1e-9))
+
+
+def conserved_fraction_bp(num_layers: int, stride: int, step_ratio_bp: int,
+                          first_ratio_bp: int = 5000) -> int:
+    """C of Eq. 9 as realised by the schedule: the last layer's keep fraction."""
+    s = Schedule(num_layers=num_layers, num_visual=10000, stride=stride,
+                 step_ratio_bp=step_ratio_bp, tau=1.0, first_ratio_bp=first_ratio_bp)
+    return s.keep_bp(num_layers - 1)
+
+
+# --------------------------------------------------------------------------
+# Attention of the current (last) query, Eq. 2 restricted to its last row.
+# --------------------------------------------------------------------------
+def attend(q: np.ndarray, K: np.ndarray, V: np.ndarray):
+    """Softmax attention of one query per head over all cached rows.
+
+    q [H, D], K [H, T, D], V [H, T, D] (float64).  Returns (out [H, D],
+    p [H, T]): p is the last row of A = Softmax((QK^T + M)/sqrt(d)); the last
+    row of a causal mask sees every position, itself included.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    d = q.shape[-1]
+    logits = np.matmul(K, q[:, :, None])[:, :, 0] / math.sqrt(d)       # [H, T]
+    logits = logits - logits.max(axis=1, keepdims=True)
+    e = np.exp(logits)
+    p = e / e.sum(axis=1, keepdims=True)
+    out = np.matmul(p[:, None, :], V)[:, 0, :]                         # [H, D]
+    return out, p
+
+
+def visual_mass(p: np.ndarray, vis_begin: int, n_vis: int) -> np.ndarray:
+    """alpha: the query's attention on each visual token, summed over heads."""
+    return p[:, vis_begin:vis_begin + n_vis].sum(axis=0)
+
+
+def select_top(scores: np.ndarray, ids: np.ndarray, k: int) -> np.ndarray:
+    """Top(G, alpha) of Eq. 3: positions of the k highest scores.
+
+    Equal scores are ordered by lower original visual index `ids`.  Returns the
+    kept positions in ascending position order.
+    """
+    n = len(scores)
+    k = max(0, min(int(k), n))
+    order = np.lexsort((np.asarray(ids), -np.asarray(scores, dtype=np.float64)))
+    return np.sort(order[:k])
+
+
+# --------------------------------------------------------------------------
+# Per-(sequence, layer) cache state: rows [S | V_kept | I | O_1..O_t].
+# --------------------------------------------------------------------------
+@dataclass
+class LayerCache:
+    K_sys: np.ndarray                 # [H, sys, D]
+    V_sys: np.ndarray
+    K_vis: np.ndarray                 # [H, n_cur, D]
+    V_vis: np.ndarray
+    ids: np.ndarray                   # [n_cur] original visual index of each kept row
+    K_txt: np.ndarray                 # [H, text + generated, D]
+    V_txt: np.ndarray
+    last_mass: np.ndarray = field(default_factory=lambda: np.zeros(0))
+
+    @property
+    def n_cur(self) -> int:
+        return int(self.ids.shape[0])
+
+    def rows(self):
+        K = np.concatenate([self.K_sys, self.K_vis, self.K_txt], axis=1)
+        V = np.concatenate([self.V_sys, self.V_vis, self.V_txt], axis=1)
+        return K, V
+
+    def keep_ids(self, kept_ids) -> None:
+        """Adopt a given kept set (teacher forcing); order of `ids` is preserved."""
+        kept = set(int(i) for i in kept_ids)
+        pos = np.array([j for j, i in enumerate(self.ids) if int(i) in kept], dtype=np.int64)
+        self.K_vis = self.K_vis[:, pos]
+        self.V_vis = self.V_vis[:, pos]
+        self.ids = self.ids[pos]
+
+
+def prefill_select(q_last, K, V, sys_len: int, num_visual: int, n_keep: int):
+    """Prefill half of Algorithm 3 for one (sequence, layer).
+
+    K, V [H, T0, D] hold the prompt rows [S | V | I]; q_last [H, D] is the last
+    prompt token's query.  Attends over the whole prompt, scores the visual
+    tokens, keeps the n_keep best (Eq. 3) and builds the cache.
+    Returns (out [H, D], mass [num_visual], cache).
+    """
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    out, p = attend(q_last, K, V)
+    mass = visual_mass(p, sys_len, num_visual)
+    ids_all = np.arange(num_visual, dtype=np.int64)
+    kept = select_top(mass, ids_all, n_keep)
+    v0, v1 = sys_len, sys_len + num_visual
+    cache = LayerCache(
+        K_sys=K[:, :v0].copy(), V_sys=V[:, :v0].copy(),
+        K_vis=K[:, v0:v1][:, kept].copy(), V_vis=V[:, v0:v1][:, kept].copy(),
+        ids=ids_all[kept].copy(),
+        K_txt=K[:, v1:].copy(), V_txt=V[:, v1:].copy(),
+        last_mass=mass,
+    )
+    return out, mass, cache
+
+
+def decode_step(cache: LayerCache, q, k_new, v_new, n_target: int):
+    """Decode half of Algorithm 3 with Eq. 7 for one (sequence, layer), one step.
+
+    Appends the new token's key/value, attends over every cached row, scores
+    the current visual rows and, if the schedule asks for fewer rows than are
+    held, keeps the n_target best and evicts the rest.
+    Returns (out [H, D], mass over the visual rows held BEFORE the eviction,
+    ids held before the eviction).
+    """
+    k_new = np.asarray(k_new, dtype=np.float64)
+    v_new = np.asarray(v_new, dtype=np.float64)
+    cache.K_txt = np.concatenate([cache.K_txt, k_new[:, None, :]], axis=1)
+    cache.V_txt = np.concatenate([cache.V_txt, v_new[:, None, :]], axis=1)
+    K, V = cache.rows()
+    out, p = attend(q, K, V)
+    n_cur = cache.n_cur
+    mass = visual_mass(p, cache.K_sys.shape[1], n_cur)
+    ids_before = cache.ids.copy()
+    n_new = min(n_cur, int(n_target))
+    if n_new < n_cur:
+        kept = select_top(mass, cache.ids, n_new)
+        cache.K_vis = cache.K_vis[:, kept]
+        cache.V_vis = cache.V_vis[:, kept]
+        cache.ids = cache.ids[kept]
+    cache.last_mass = mass
+    return out, mass, ids_before
+
+
+def boundary_scores(mass: np.ndarray, ids: np.ndarray, k: int):
+    """(s_k, s_{k+1}): the k-th and (k+1)-th scores in selection order (None if absent)."""
+    n = len(mass)
+    order = np.lexsort((np.asarray(ids), -np.asarray(mass, dtype=np.float64)))
+    s_k = float(mass[order[k - 1]]) if 1 <= k <= n else None
+    s_k1 = float(mass[order[k]]) if 0 <= k < n else None
+    return s_k, s_k1

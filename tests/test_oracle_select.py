@@ -1,0 +1,76 @@
+"""Pins for Top(G, alpha) (Eq. 3) with the lower-index tie-break, and for cache bookkeeping."""
+import numpy as np
+import pytest
+
+from oracle.st3_oracle import select_top, boundary_scores, prefill_select, decode_step
+
+
+def _exhaustive(scores, ids, k):
+    """i is kept iff fewer than k tokens beat it (higher score, or equal score and lower id)."""
+    n = len(scores)
+    keep = []
+    for i in range(n):
+        beat = sum(1 for j in range(n)
+                   if scores[j] > scores[i] or (scores[j] == scores[i] and ids[j] < ids[i]))
+        if beat < k:
+            keep.append(i)
+    return np.array(keep, dtype=np.int64)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_matches_exhaustive_definition_with_ties(seed):
+    r = np.random.default_rng(seed)
+    n = int(r.integers(1, 40))
+    scores = r.integers(0, 5, size=n).astype(np.float64) / 4.0     # many exact ties
+    ids = r.permutation(100)[:n]
+    for k in range(0, n + 1):
+        assert np.array_equal(select_top(scores, ids, k), _exhaustive(scores, ids, k))
+
+
+def test_all_equal_keeps_lowest_ids_and_extremes():
+    ids = np.array([9, 2, 7, 4, 0, 5])
+    s = np.full(6, 0.25)
+    kept = select_top(s, ids, 3)
+    assert sorted(ids[kept].tolist()) == [0, 2, 4]
+    assert len(select_top(s, ids, 0)) == 0
+    assert np.array_equal(select_top(s, ids, 6), np.arange(6))
+    assert np.array_equal(select_top(s, ids, 99), np.arange(6))
+
+
+def test_no_ties_equals_sort():
+    r = np.random.default_rng(11)
+    s = r.random(50)
+    kept = select_top(s, np.arange(50), 20)
+    assert set(kept.tolist()) == set(np.argsort(-s)[:20].tolist())
+    sk, sk1 = boundary_scores(s, np.arange(50), 20)
+    srt = np.sort(s)[::-1]
+    assert sk == srt[19] and sk1 == srt[20]
+
+
+def test_prefill_and_decode_bookkeeping():
+    r = np.random.default_rng(12)
+    H, D, sys_len, nv, text = 2, 4, 3, 10, 4
+    T0 = sys_len + nv + text
+    K, V = r.standard_normal((H, T0, D)), r.standard_normal((H, T0, D))
+    q = r.standard_normal((H, D))
+    out, mass, c = prefill_select(q, K, V, sys_len, nv, 6)
+    assert c.n_cur == 6 and mass.shape == (nv,)
+    # kept rows are bit-identical to the source rows their ids name
+    assert np.array_equal(c.K_vis, K[:, sys_len + c.ids]) and np.array_equal(c.V_vis, V[:, sys_len + c.ids])
+    assert np.array_equal(c.K_sys, K[:, :sys_len]) and np.array_equal(c.K_txt, K[:, sys_len + nv:])
+    assert set(c.ids.tolist()) == set(np.argsort(-mass)[:6].tolist())
+    kn, vn = r.standard_normal((H, D)), r.standard_normal((H, D))
+    ids0 = c.ids.copy()
+    out1, m1, before = decode_step(c, r.standard_normal((H, D)), kn, vn, 4)
+    assert np.array_equal(before, ids0) and m1.shape == (6,)
+    assert c.n_cur == 4 and set(c.ids.tolist()) <= set(ids0.tolist())
+    assert c.K_txt.shape[1] == text + 1 and np.array_equal(c.K_txt[:, -1], kn)
+    assert np.array_equal(c.K_vis, K[:, sys_len + c.ids])
+    # a target above the current count never grows the cache
+    decode_step(c, r.standard_normal((H, D)), kn, vn, 9)
+    assert c.n_cur == 4
+    # empty visual span is legal (beta = 0)
+    decode_step(c, r.standard_normal((H, D)), kn, vn, 0)
+    assert c.n_cur == 0
+    o, m, _ = decode_step(c, r.standard_normal((H, D)), kn, vn, 0)
+    assert m.shape == (0,) and np.all(np.isfinite(o))

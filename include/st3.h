@@ -1,0 +1,174 @@
+/*
+ * st3.h -- C ABI of the ST^3 decode-attention + visual-token-trimming library (sm_100a).
+ *
+ * The library keeps, per decoder layer and per sequence, a key/value cache whose rows are
+ * [system | kept visual | instruction text | generated] tokens (Eq. 1 of the ST^3 paper:
+ * X = [S, V, I, O]).  One decode step, for every requested layer and sequence,
+ *   1. appends the new token's key/value row,
+ *   2. computes the current query's softmax attention over every cached row (Eq. 2, last row),
+ *   3. accumulates each visual token's attention probability over heads (the score alpha
+ *      of Sec. 3.2),
+ *   4. if the retention schedule asks for fewer visual rows than are held, keeps the
+ *      top-scoring ones (Eq. 3, ties toward the lower original visual index), and
+ *   5. compacts the kept K/V rows in place.
+ * The retention schedule is PVTP per layer (Sec. 3.2, Algorithm 1, Eq. 9) times VTA per step
+ * (Sec. 3.3, Eq. 7 and Eq. 8).
+ *
+ * Conventions for every entry point
+ *   - "dev" pointers are CUDA device pointers, "host" pointers are ordinary host memory.
+ *   - All device pointers must be 16-byte aligned; tensors are dense, row-major, in the
+ *     element type named by st3_config.dtype.
+ *   - The caller owns every buffer, including the workspace; the library allocates no device
+ *     memory and frees only its own host-side context.
+ *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as void*) and the call
+ *     returns without waiting for it unless stated otherwise.  Calls on one context must be
+ *     issued in program order; buffers must stay valid until the enqueued work has finished.
+ *   - Errors are reported through the return code.  Problems detected on the device (a count
+ *     that disagrees with the schedule, a non-finite score, a copy that never arrived) are
+ *     OR-ed into a device status word read with st3_get_status.  The library never aborts,
+ *     throws or traps.
+ */
+#ifndef ST3_H_
+#define ST3_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct st3_ctx st3_ctx;
+
+typedef enum {
+  ST3_OK = 0,
+  ST3_ERR_INVALID_ARG = 1,         /* null / misaligned pointer, out-of-range value            */
+  ST3_ERR_WORKSPACE_TOO_SMALL = 2, /* workspace smaller than st3_workspace_size reports        */
+  ST3_ERR_BAD_STATE = 3,           /* call order violated (decode before prefill, step gap)    */
+  ST3_ERR_CAPACITY = 4,            /* text length or step beyond the configured maximum        */
+  ST3_ERR_CUDA = 5,                /* a CUDA runtime call failed                               */
+  ST3_ERR_DEVICE_CHECK = 6,        /* st3_get_status found a non-zero device status word       */
+  ST3_ERR_UNSUPPORTED = 7          /* shape outside what the kernels are built for             */
+} st3_status;
+
+typedef enum { ST3_F32 = 0, ST3_BF16 = 1 } st3_dtype;
+
+/* Attenuation function beta(t) of VTA: Eq. 8 (cosine) and the two alternatives of Sec. 4.4. */
+typedef enum { ST3_ANNEAL_COSINE = 0, ST3_ANNEAL_NONE = 1, ST3_ANNEAL_LINEAR = 2, ST3_ANNEAL_EXP = 3 } st3_anneal;
+
+/* Bits of the device status word. */
+enum {
+  ST3_DEV_COUNT_MISMATCH = 1,  /* a layer's device-side visual count differs from the schedule */
+  ST3_DEV_NONFINITE = 2,       /* a visual score was NaN/Inf/negative                          */
+  ST3_DEV_COPY_TIMEOUT = 4,    /* an asynchronous shared-memory copy did not complete in time  */
+  ST3_DEV_RANGE = 8            /* an index left its buffer (the access was skipped)            */
+};
+
+typedef struct {
+  int32_t num_layers;        /* L: decoder layers (<= 64)                                       */
+  int32_t num_heads;         /* H: multi-head attention, kv heads == query heads (<= 128)       */
+  int32_t head_dim;          /* D: 64 or 128                                                    */
+  int32_t dtype;             /* st3_dtype of q/k/v/out and of the cache                          */
+  int32_t batch;             /* B: independent sequences                                        */
+  int32_t sys_len;           /* |S|: system-prompt tokens in front of the visual span           */
+  int32_t num_visual;        /* |V| at the input of layer 0                                     */
+  int32_t max_text_len;      /* capacity for |I| per sequence                                   */
+  int32_t max_decode_steps;  /* capacity for |O|                                                */
+  int32_t first_prune_layer; /* 3: "avoid pruning tokens in the first three layers" (Sec. 3.2)  */
+  int32_t stride;            /* S: prune at layers first, first+S, ... (Algorithm 1)            */
+  int32_t first_ratio_bp;    /* P in basis points of |V|; the paper sets 50% = 5000 (Eq. 9)     */
+  int32_t step_ratio_bp;     /* R in basis points of |V| removed at each later pruning layer    */
+  int32_t anneal;            /* st3_anneal                                                      */
+  int32_t disable_trim;      /* 1: same kernels, nothing is ever evicted (full-KV comparison)   */
+  int32_t rows_per_chunk;    /* cache rows one thread block attends over (<= 256); 0 = choose   */
+  double tau;                /* Eq. 8: beta = cos(t*pi/(2 tau)) for t < tau, else 0             */
+  double sigma;              /* only ST3_ANNEAL_EXP: beta = exp(-t/sigma)                       */
+} st3_config;
+
+/* Scheduled visual-row count n(l, t) of layer `layer` after decode step `step` (0 = after
+ * prefill).  Pure host function.  PVTP: layers below first_prune_layer keep everything; layer l
+ * in stage k = (l - first)/S keeps floor(|V| * (1 - P - k R)) (Eq. 9 read additively, the
+ * reading that reproduces the paper's printed (S, R, C) tables).  VTA: n(l,t) =
+ * floor(n(l,0) * beta(t)) (Eq. 7, Eq. 8).  Returns -1 on an invalid argument. */
+int32_t st3_schedule_count(const st3_config* cfg, int32_t layer, int32_t step);
+
+/* Bytes of device workspace st3_create needs for `cfg` (host call, no CUDA work). */
+st3_status st3_workspace_size(const st3_config* cfg, size_t* bytes);
+
+/* Builds a context over a caller-owned device workspace (256-byte aligned, `bytes` long, on the
+ * current device).  Host-side set-up plus one cudaMemsetAsync of the bookkeeping area on the
+ * default stream, which is synchronised before returning.  *out is NULL on failure. */
+st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, st3_ctx** out);
+
+/* Prefill half of Algorithm 3 for layers [layer_begin, layer_begin+layer_count): ingests the
+ * prompt's K/V rows into the cache, attends with the last prompt token's query over the whole
+ * prompt, scores the visual tokens and keeps the n(l,0) best (Eq. 3).
+ *   q_last   dev  [layer_count][B][H][D]
+ *   k, v     dev  [layer_count][B][H][t0_max][D], t0_max = sys_len + num_visual + max_text_len,
+ *                 rows in the order [S | V | I]; rows past a sequence's text length are ignored
+ *   text_len host [B], each in [1, max_text_len]; read before the call returns; must be the
+ *                 same values for every layer range of one generation
+ *   out      dev  [layer_count][B][H][D] attention output of the last prompt token
+ * Resets the step counter of those layers to 0. */
+st3_status st3_prefill_select(st3_ctx* ctx, int32_t layer_begin, int32_t layer_count,
+                              const void* q_last, const void* k, const void* v,
+                              const int32_t* text_len, void* out, void* cuda_stream);
+
+/* One decode step (Algorithm 3's decode half with Eq. 7) for the given layers: append, attend,
+ * score, select, compact.  `step` counts from 1 and must be the previous step of each of these
+ * layers plus one (else ST3_ERR_BAD_STATE); step > max_decode_steps gives ST3_ERR_CAPACITY.
+ *   q, k_new, v_new  dev [layer_count][B][H][D]   query and new key/value row of this step
+ *   out              dev [layer_count][B][H][D]   attention output
+ * After the call the cache of layer l holds n(l, step) visual rows. */
+st3_status st3_decode_step(st3_ctx* ctx, int32_t step, int32_t layer_begin, int32_t layer_count,
+                           const void* q, const void* k_new, const void* v_new, void* out,
+                           void* cuda_stream);
+
+/* Same step with HOST buffers (pinned memory recommended): the library copies q/k_new/v_new to
+ * staging areas inside its workspace, runs the step and copies `out` back, all on the stream.
+ * The host buffers must stay untouched until the stream has passed the call. */
+st3_status st3_decode_step_host(st3_ctx* ctx, int32_t step, int32_t layer_begin, int32_t layer_count,
+                                const void* q_host, const void* k_new_host, const void* v_new_host,
+                                void* out_host, void* cuda_stream);
+
+/* Observability: copies layer `layer`'s kept original visual indices (ids dev [B][num_visual],
+ * first count[b] entries valid, cache order), counts (count dev [B]) and, if mass != NULL, the
+ * score computed at each token's most recent selection indexed by ORIGINAL visual index
+ * (mass dev [B][num_visual]; entries of tokens never scored are 0). */
+st3_status st3_get_kept(st3_ctx* ctx, int32_t layer, int32_t* ids, int32_t* count, float* mass,
+                        void* cuda_stream);
+
+/* Copies cache rows of (layer, sequence b, head h) to dev buffers of the cache dtype, for tests:
+ * k_vis/v_vis [num_visual][D] (first count rows valid), k_txt/v_txt [cap][D] with
+ * cap = sys_len + max_text_len + max_decode_steps, rows [S | I | O].  Any pointer may be NULL. */
+st3_status st3_get_rows(st3_ctx* ctx, int32_t layer, int32_t b, int32_t h, void* k_vis, void* v_vis,
+                        void* k_txt, void* v_txt, void* cuda_stream);
+
+/* Synchronises the stream last used by this context and returns the device status word through
+ * *word (host).  Returns ST3_ERR_DEVICE_CHECK if it is non-zero. */
+st3_status st3_get_status(st3_ctx* ctx, int32_t* word);
+
+/* Visual + non-visual K/V rows currently held, summed over layers and sequences (host
+ * bookkeeping, exact by the schedule); multiply by 2*H*D*sizeof(element) for bytes. */
+st3_status st3_rows_held(st3_ctx* ctx, int64_t* visual_rows, int64_t* other_rows);
+
+/* Kernel timing for roofline reports.  While enabled, every prefill/decode call records CUDA
+ * events around its attention kernel and around its select/compact kernel on the call's stream.
+ * st3_profile_read synchronises, returns the accumulated milliseconds and launch counts since
+ * enabling (any pointer may be NULL) and clears them. */
+st3_status st3_profile_enable(st3_ctx* ctx, int32_t on);
+st3_status st3_profile_read(st3_ctx* ctx, double* attn_ms, double* finish_ms, int64_t* attn_launches,
+                            int64_t* finish_launches);
+
+/* Total kernels this context has launched so far (host counter). */
+int64_t st3_launch_count(const st3_ctx* ctx);
+
+const char* st3_status_string(st3_status s);
+
+/* Frees the host-side context.  Does not synchronise and does not touch the workspace. */
+st3_status st3_destroy(st3_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ST3_H_ */

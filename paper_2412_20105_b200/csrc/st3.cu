@@ -1,0 +1,1025 @@
+// ST^3 decode-step attention over a trimmed visual KV cache: sm_100a kernels and the C ABI.
+//
+// Cache layout (device, caller's workspace).  For every (layer l, sequence b, head h) one block
+//   [ K_vis : Nv x D ][ V_vis : Nv x D ][ K_txt : cap x D ][ V_txt : cap x D ]
+// with cap = sys_len + max_text_len + max_decode_steps.  The visual rows live in their own
+// region so that evicting them never shifts system / text / generated rows; the text region
+// holds [S | I | O_1.. ] in order.  ids[l][b][i] is the ORIGINAL visual index of visual row i.
+//
+// One step = two launches:
+//   st3_attend_kernel   one thread block per (l, b, head, row chunk).  The chunk's K and V rows
+//                       are brought into shared memory with bulk asynchronous copies
+//                       (cp.async.bulk + mbarrier, 16 KB pieces), the block computes the chunk's
+//                       logits, its local softmax statistics (m, l) and its un-normalised
+//                       output, and - for layers that evict at this step - stores the raw logits
+//                       of visual rows.  The block that owns the newest text row also appends it.
+//   st3_finish_kernel   one block per (l, b): merges the chunk partials of every head into the
+//                       attention output, turns the raw logits into head-summed probabilities
+//                       (the visual score alpha), radix-selects the rows to keep (ties toward the
+//                       lower original index) and fills the holes among the first n_new rows with
+//                       the kept rows of the tail, so the kept rows end up dense and the minimum
+//                       number of rows moves.
+// The work decomposition is computed on the host from the schedule (row counts are a pure
+// function of layer and step), so no table is uploaded per step.
+#include "st3.h"
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kPieceRows = 64;  // rows per bulk copy / mbarrier
+constexpr int kMaxChunkRows = 256;
+constexpr int kMaxPieces = kMaxChunkRows / kPieceRows;
+constexpr int kMaxLayers = 64;
+constexpr int kMaxHeads = 128;
+constexpr int kMaxVisual = 8192;
+constexpr long long kWaitCycles = 4000000000LL;  // ~2 s: bound on any wait for an async copy
+
+struct StepParams {
+  const void* q;
+  const void* k_new;
+  const void* v_new;
+  void* out;
+  void* cache;
+  float* part_ml;        // [item*H + h][2]  (m, l) in the log2 domain
+  float* part_acc;       // [item*H + h][D]  un-normalised output
+  float* logits;         // [l][b][h][Nv]    raw log2-domain logits of visual rows
+  float* mass_by_id;     // [l][b][Nv]
+  int* ids;              // [l][b][Nv]
+  int* n_cur;            // [l][b]
+  const int* text_len;   // [b]
+  int* status;
+  long long lbh_stride;  // elements per (l, b, h) cache block
+  int layer_begin, layer_count, B, H;
+  int sys_len, Nv, cap_txt, step, append;
+  int ct;                   // text chunks per (l, b, h), the same for every sequence
+  int chunk_rows;           // shared-memory tile capacity in rows
+  int cvp[kMaxLayers + 1];  // prefix sum of visual chunks per layer (relative layer index)
+  int ncur[kMaxLayers];     // visual rows held before this step (host's schedule bookkeeping)
+  int ntgt[kMaxLayers];     // visual rows to hold after this step
+};
+
+// ------------------------------------------------------------------------------------------
+// PTX helpers: mbarrier + bulk asynchronous global->shared copy
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void bulk_g2s(void* dst_smem, const void* src_gmem, uint32_t bytes, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+          smem_u32(dst_smem)),
+      "l"(src_gmem), "r"(bytes), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after kWaitCycles, records it in the status word and lets the block run
+// to completion on whatever is in shared memory (the result is then flagged invalid).
+__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
+  if (mbar_try_wait(bar, parity)) return;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > kWaitCycles) {
+      atomicOr(status, ST3_DEV_COPY_TIMEOUT);
+      return;
+    }
+  }
+}
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// 16 bytes -> EPL floats
+__device__ __forceinline__ void unpack16(const uint4& v, float (&f)[8]) {  // bf16 x 8
+  f[0] = __uint_as_float(v.x << 16);
+  f[1] = __uint_as_float(v.x & 0xffff0000u);
+  f[2] = __uint_as_float(v.y << 16);
+  f[3] = __uint_as_float(v.y & 0xffff0000u);
+  f[4] = __uint_as_float(v.z << 16);
+  f[5] = __uint_as_float(v.z & 0xffff0000u);
+  f[6] = __uint_as_float(v.w << 16);
+  f[7] = __uint_as_float(v.w & 0xffff0000u);
+}
+__device__ __forceinline__ void unpack16(const uint4& v, float (&f)[4]) {  // f32 x 4
+  f[0] = __uint_as_float(v.x);
+  f[1] = __uint_as_float(v.y);
+  f[2] = __uint_as_float(v.z);
+  f[3] = __uint_as_float(v.w);
+}
+__device__ __forceinline__ void store_out(float* p, float v) { *p = v; }
+__device__ __forceinline__ void store_out(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Which (relative layer, sequence, chunk) a flat item index names.  Items are ordered by layer,
+// then sequence, then chunk (visual chunks first, then text chunks).
+struct Item {
+  int l_rel, b, c, cv;
+};
+__device__ __forceinline__ Item decode_item(const StepParams& p, int item) {
+  int lo = 0, hi = p.layer_count - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (p.B * (p.cvp[mid] + mid * p.ct) <= item) lo = mid; else hi = mid - 1;
+  }
+  Item it;
+  it.l_rel = lo;
+  it.cv = p.cvp[lo + 1] - p.cvp[lo];
+  const int off = item - p.B * (p.cvp[lo] + lo * p.ct);
+  const int per = it.cv + p.ct;
+  it.b = off / per;
+  it.c = off - it.b * per;
+  return it;
+}
+
+// ------------------------------------------------------------------------------------------
+// Attention partials (Eq. 2, last row) + raw visual logits + KV append
+// ------------------------------------------------------------------------------------------
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads) st3_attend_kernel(const StepParams p) {
+  constexpr int EPL = 16 / sizeof(T);  // elements per 16-byte lane load
+  constexpr int LPR = D / EPL;         // lanes per row
+  constexpr int RPW = 32 / LPR;        // rows per warp instruction
+  constexpr int ROWB = D * sizeof(T);
+  static_assert(LPR <= 32 && RPW >= 1, "row must fit one warp instruction");
+
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ float s_red[kWarps * D];
+  __shared__ float s_stat[kWarps];
+  __shared__ __align__(8) uint64_t s_bar[2 * kMaxPieces];
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int H = p.H;
+  const int h = blockIdx.x % H;
+  const int item = blockIdx.x / H;
+  const Item it = decode_item(p, item);
+  const int l = p.layer_begin + it.l_rel, b = it.b;
+  const bool is_vis = it.c < it.cv;
+
+  // rows of this chunk
+  int seg_rows, nchunk, ci;
+  if (is_vis) {
+    seg_rows = p.ncur[it.l_rel]; nchunk = it.cv; ci = it.c;
+  } else {
+    seg_rows = p.sys_len + __ldg(p.text_len + b) + p.step; nchunk = p.ct; ci = it.c - it.cv;
+  }
+  const int rows_per = (seg_rows + nchunk - 1) / nchunk;
+  const int r0 = ci * rows_per;
+  const int r1 = min(seg_rows, r0 + rows_per);
+  const int nrows = r1 - r0;
+  const long long slot = (long long)item * H + h;
+  if (nrows <= 0 || nrows > p.chunk_rows) {  // empty chunk (ragged split); uniform for the block
+    if (nrows > p.chunk_rows && tid == 0) atomicOr(p.status, ST3_DEV_RANGE);
+    if (tid == 0) { p.part_ml[2 * slot] = -INFINITY; p.part_ml[2 * slot + 1] = 0.f; }
+    if (tid < D) p.part_acc[slot * D + tid] = 0.f;
+    return;
+  }
+  const bool has_new = !is_vis && p.append && r1 == seg_rows;  // this chunk ends on the newest row
+  const int nbulk = nrows - (has_new ? 1 : 0);
+
+  const long long lbh = ((long long)l * p.B + b) * H + h;
+  T* blk = reinterpret_cast<T*>(p.cache) + lbh * p.lbh_stride;
+  T* gK = is_vis ? blk : blk + 2LL * p.Nv * D;
+  T* gV = gK + (is_vis ? (long long)p.Nv * D : (long long)p.cap_txt * D);
+
+  unsigned char* sK = smem;
+  unsigned char* sV = smem + (size_t)p.chunk_rows * ROWB;
+  float* s_log = reinterpret_cast<float*>(sV + (size_t)p.chunk_rows * ROWB);
+
+  if (tid == 0) {
+    const int npiece = (nbulk + kPieceRows - 1) / kPieceRows;
+    for (int i = 0; i < npiece; ++i) { mbar_init(&s_bar[i], 1); mbar_init(&s_bar[kMaxPieces + i], 1); }
+    mbar_fence_init();
+    for (int kv = 0; kv < 2; ++kv) {
+      const unsigned char* g = reinterpret_cast<const unsigned char*>(kv ? gV : gK) + (size_t)r0 * ROWB;
+      unsigned char* s = kv ? sV : sK;
+      for (int i = 0; i < npiece; ++i) {
+        const int rows = min(kPieceRows, nbulk - i * kPieceRows);
+        const uint32_t bytes = (uint32_t)rows * ROWB;
+        uint64_t* bar = &s_bar[kv * kMaxPieces + i];
+        mbar_expect_tx(bar, bytes);
+        bulk_g2s(s + (size_t)i * kPieceRows * ROWB, g + (size_t)i * kPieceRows * ROWB, bytes, bar);
+      }
+    }
+  }
+
+  const int sub = lane / LPR;  // which of the RPW rows of a warp instruction
+  const int lir = lane % LPR;  // 16-byte column inside the row
+  const long long qoff = (((long long)it.l_rel * p.B + b) * H + h) * D;
+
+  // query, pre-scaled by log2(e)/sqrt(D) so that probabilities are exp2(logit - max)
+  float qf[EPL];
+  {
+    const uint4 qv = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.q) + qoff) + lir);
+    unpack16(qv, qf);
+    const float sc = 1.4426950408889634f * rsqrtf((float)D);
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) qf[e] *= sc;
+  }
+  // newest row: comes from the step's inputs, goes to the cache and into the tile
+  if (has_new && tid < 2 * LPR) {
+    const int kv = tid / LPR, c = tid % LPR;
+    const T* src = reinterpret_cast<const T*>(kv ? p.v_new : p.k_new) + qoff;
+    const uint4 val = __ldg(reinterpret_cast<const uint4*>(src) + c);
+    T* dstg = (kv ? gV : gK) + (long long)(seg_rows - 1) * D;
+    reinterpret_cast<uint4*>(dstg)[c] = val;
+    *reinterpret_cast<uint4*>((kv ? sV : sK) + (size_t)(nrows - 1) * ROWB + c * 16) = val;
+  }
+  __syncthreads();  // barrier inits and the newest row are visible
+
+  // ---- K pass: logits ----
+  for (int base = 0; base < nrows; base += kPieceRows) {
+    if (base < nbulk) mbar_wait(&s_bar[base / kPieceRows], 0, p.status);
+    const int pend = min(nrows, base + kPieceRows);
+#pragma unroll 2
+    for (int rb = base + warp * RPW; rb < pend; rb += kWarps * RPW) {
+      const int r = rb + sub;
+      float acc = 0.f;
+      if (r < pend) {
+        const uint4 kvv = *reinterpret_cast<const uint4*>(sK + (size_t)r * ROWB + lir * 16);
+        float kf[EPL];
+        unpack16(kvv, kf);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc = fmaf(qf[e], kf[e], acc);
+      }
+#pragma unroll
+      for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (r < pend && lir == 0) s_log[r] = acc;
+    }
+  }
+  __syncthreads();
+
+  // ---- chunk softmax statistics ----
+  float mloc = -INFINITY;
+  for (int r = tid; r < nrows; r += kThreads) mloc = fmaxf(mloc, s_log[r]);
+  mloc = warp_max(mloc);
+  if (lane == 0) s_stat[warp] = mloc;
+  __syncthreads();
+  float m = s_stat[0];
+#pragma unroll
+  for (int w = 1; w < kWarps; ++w) m = fmaxf(m, s_stat[w]);
+  __syncthreads();
+  const bool want_logits = is_vis && p.ntgt[it.l_rel] < p.ncur[it.l_rel];
+  float* glog = p.logits + lbh * p.Nv + r0;
+  float lsum = 0.f;
+  for (int r = tid; r < nrows; r += kThreads) {
+    const float s = s_log[r];
+    if (want_logits) glog[r] = s;
+    const float pr = fast_exp2(s - m);
+    s_log[r] = pr;
+    lsum += pr;
+  }
+  lsum = warp_sum(lsum);
+  if (lane == 0) s_stat[warp] = lsum;
+  __syncthreads();  // also publishes the probabilities in s_log
+  if (tid == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) t += s_stat[w];
+    p.part_ml[2 * slot] = m;
+    p.part_ml[2 * slot + 1] = t;
+  }
+
+  // ---- V pass: un-normalised output ----
+  float acc[EPL];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  for (int base = 0; base < nrows; base += kPieceRows) {
+    if (base < nbulk) mbar_wait(&s_bar[kMaxPieces + base / kPieceRows], 0, p.status);
+    const int pend = min(nrows, base + kPieceRows);
+#pragma unroll 2
+    for (int rb = base + warp * RPW; rb < pend; rb += kWarps * RPW) {
+      const int r = rb + sub;
+      if (r < pend) {
+        const float pr = s_log[r];
+        const uint4 vv = *reinterpret_cast<const uint4*>(sV + (size_t)r * ROWB + lir * 16);
+        float vf[EPL];
+        unpack16(vv, vf);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) acc[e] = fmaf(pr, vf[e], acc[e]);
+      }
+    }
+  }
+#pragma unroll
+  for (int o = LPR; o < 32; o <<= 1) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+  }
+  if (lane < LPR) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) s_red[warp * D + lir * EPL + e] = acc[e];
+  }
+  __syncthreads();
+  if (tid < D) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) t += s_red[w * D + tid];
+    p.part_acc[slot * D + tid] = t;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Merge partials, visual scores, top-k (Eq. 3), in-place compaction (Eq. 7's eviction)
+// ------------------------------------------------------------------------------------------
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p) {
+  constexpr int ROWB = D * sizeof(T);
+  constexpr int VPR = ROWB / 16;  // 16-byte vectors per row
+  extern __shared__ __align__(16) unsigned char smem[];
+  __shared__ float s_M[kMaxHeads];
+  __shared__ float s_invL[kMaxHeads];
+  __shared__ int s_hist[256];
+  __shared__ int s_scan[kWarps];
+  __shared__ int s_sel[3];  // digit, count above, count in bin
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int B = p.B, H = p.H, Nv = p.Nv;
+  const int l_rel = blockIdx.x / B, b = blockIdx.x % B;
+  const int l = p.layer_begin + l_rel;
+  const int cv = p.cvp[l_rel + 1] - p.cvp[l_rel];
+  const int nit = cv + p.ct;
+  const long long item0 = (long long)B * (p.cvp[l_rel] + l_rel * p.ct) + (long long)b * nit;
+
+  // ---- merge the chunk partials of every head ----
+  for (int h = warp; h < H; h += kWarps) {
+    float M = -INFINITY;
+    for (int s = lane; s < nit; s += 32) M = fmaxf(M, p.part_ml[2 * ((item0 + s) * H + h)]);
+    M = warp_max(M);
+    float L = 0.f;
+    for (int s = lane; s < nit; s += 32) {
+      const long long slot = (item0 + s) * H + h;
+      L += p.part_ml[2 * slot + 1] * fast_exp2(p.part_ml[2 * slot] - M);
+    }
+    L = warp_sum(L);
+    float o[D / 32];
+#pragma unroll
+    for (int j = 0; j < D / 32; ++j) o[j] = 0.f;
+    for (int s = 0; s < nit; ++s) {
+      const long long slot = (item0 + s) * H + h;
+      const float w = fast_exp2(p.part_ml[2 * slot] - M);
+#pragma unroll
+      for (int j = 0; j < D / 32; ++j) o[j] = fmaf(w, p.part_acc[slot * D + lane + 32 * j], o[j]);
+    }
+    const float invL = 1.f / L;
+    T* out = reinterpret_cast<T*>(p.out) + (((long long)l_rel * B + b) * H + h) * D;
+#pragma unroll
+    for (int j = 0; j < D / 32; ++j) store_out(out + lane + 32 * j, o[j] * invL);
+    if (lane == 0) { s_M[h] = M; s_invL[h] = invL; }
+  }
+  __syncthreads();
+
+  const long long lb = (long long)l * B + b;
+  const int n_cur = p.n_cur[lb];
+  if (n_cur != p.ncur[l_rel]) {  // host bookkeeping and device state disagree: flag, do not touch
+    if (tid == 0) atomicOr(p.status, ST3_DEV_COUNT_MISMATCH);
+    return;
+  }
+  const int k = min(n_cur, p.ntgt[l_rel]);
+  if (k >= n_cur) return;
+
+  unsigned long long* s_key = reinterpret_cast<unsigned long long*>(smem);  // [Nv]
+  int* s_hole = reinterpret_cast<int*>(smem + (size_t)Nv * 8);              // [Nv]
+  int* s_mover = s_hole + Nv;                                               // [Nv]
+  int* ids = p.ids + lb * Nv;
+  float* mass_by_id = p.mass_by_id + lb * Nv;
+
+  // ---- visual scores: probability of every visual row summed over heads ----
+  bool bad = false;
+  for (int i = tid; i < n_cur; i += kThreads) {
+    float mass = 0.f;
+    const float* lg = p.logits + lb * H * Nv + i;
+    for (int h = 0; h < H; ++h) mass += fast_exp2(lg[(long long)h * Nv] - s_M[h]) * s_invL[h];
+    if (!(mass >= 0.f) || !(mass <= 3.0e38f)) { bad = true; mass = 0.f; }
+    const int id = ids[i];
+    mass_by_id[id] = mass;
+    s_key[i] = ((unsigned long long)__float_as_uint(mass) << 32) | (unsigned long long)(0xffffffffu - (unsigned)id);
+  }
+  if (bad) atomicOr(p.status, ST3_DEV_NONFINITE);
+  __syncthreads();
+
+  // ---- radix select: the k-th largest 64-bit key (keys are unique: ids are) ----
+  unsigned long long prefix = 0ull, mask = 0ull;
+  if (k > 0) {
+    int need = k;
+    for (int shift = 56; shift >= 0; shift -= 8) {
+      s_hist[tid] = 0;
+      __syncthreads();
+      for (int i = tid; i < n_cur; i += kThreads) {
+        const unsigned long long key = s_key[i];
+        if ((key & mask) == prefix) atomicAdd(&s_hist[(int)((key >> shift) & 0xffull)], 1);
+      }
+      __syncthreads();
+      if (warp == 0) {
+        int c[8], t = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = s_hist[lane * 8 + j]; t += c[j]; }
+        int S = t;  // inclusive suffix sum over lanes (this lane and the higher ones)
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_down_sync(0xffffffffu, S, o);
+          if (lane + o < 32) S += v;
+        }
+        int above = S - t;
+        if (above < need && need <= S) {
+#pragma unroll
+          for (int j = 7; j >= 0; --j) {
+            if (above + c[j] >= need) { s_sel[0] = lane * 8 + j; s_sel[1] = above; s_sel[2] = c[j]; break; }
+            above += c[j];
+          }
+        }
+      }
+      __syncthreads();
+      const int digit = s_sel[0], above = s_sel[1], inbin = s_sel[2];
+      need -= above;
+      prefix |= (unsigned long long)digit << shift;
+      mask |= 0xffull << shift;
+      if (need == inbin) break;  // the whole bin is kept: keys >= prefix are exactly the top k
+    }
+  } else {
+    prefix = ~0ull;  // keep nothing (ids are < 2^31, so no key reaches this value)
+  }
+
+  // ---- pair every hole among the first k rows with a kept row of the tail ----
+  const int per = (n_cur + kThreads - 1) / kThreads;
+  const int i0 = min(n_cur, tid * per), i1 = min(n_cur, i0 + per);
+  int nh = 0, nm = 0;
+  for (int i = i0; i < i1; ++i) {
+    const bool keep = s_key[i] >= prefix;
+    nh += (i < k && !keep);
+    nm += (i >= k && keep);
+  }
+  const int packed = nh | (nm << 16);
+  int incl = packed;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) s_scan[warp] = incl;
+  __syncthreads();
+  int woff = 0, total = 0;
+#pragma unroll
+  for (int w = 0; w < kWarps; ++w) {
+    if (w < warp) woff += s_scan[w];
+    total += s_scan[w];
+  }
+  const int excl = woff + incl - packed;
+  int ph = excl & 0xffff, pm = excl >> 16;
+  for (int i = i0; i < i1; ++i) {
+    const bool keep = s_key[i] >= prefix;
+    if (i < k && !keep) s_hole[ph++] = i;
+    if (i >= k && keep) s_mover[pm++] = i;
+  }
+  __syncthreads();
+  const int nmove = total & 0xffff;
+  if (nmove != (total >> 16)) {  // cannot happen when exactly k keys pass the threshold
+    if (tid == 0) atomicOr(p.status, ST3_DEV_RANGE);
+    return;
+  }
+
+  // ---- move the rows (sources are rows >= k, destinations rows < k: disjoint) ----
+  unsigned char* blk0 = reinterpret_cast<unsigned char*>(p.cache) + (size_t)(lb * H) * p.lbh_stride * sizeof(T);
+  const long long nvec = (long long)nmove * H * 2 * VPR;
+  for (long long v = tid; v < nvec; v += kThreads) {
+    const int c = (int)(v % VPR);
+    long long r = v / VPR;
+    const int kv = (int)(r % 2); r /= 2;
+    const int h = (int)(r % H);
+    const int j = (int)(r / H);
+    unsigned char* base = blk0 + (size_t)h * p.lbh_stride * sizeof(T) + (size_t)kv * Nv * ROWB;
+    const uint4 val = *reinterpret_cast<const uint4*>(base + (size_t)s_mover[j] * ROWB + c * 16);
+    *reinterpret_cast<uint4*>(base + (size_t)s_hole[j] * ROWB + c * 16) = val;
+  }
+  for (int j = tid; j < nmove; j += kThreads) ids[s_hole[j]] = ids[s_mover[j]];
+  if (tid == 0) p.n_cur[lb] = k;
+}
+
+// ------------------------------------------------------------------------------------------
+// Prompt ingest: rows [S | V | I] of the caller's tensors -> cache regions
+// ------------------------------------------------------------------------------------------
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads) st3_ingest_kernel(const StepParams p, const T* __restrict__ k,
+                                                              const T* __restrict__ v, int t0_max) {
+  constexpr int VPR = D * sizeof(T) / 16;
+  const int H = p.H, B = p.B, Nv = p.Nv;
+  int y = blockIdx.y;
+  const int h = y % H; y /= H;
+  const int b = y % B;
+  const int l_rel = y / B;
+  const int l = p.layer_begin + l_rel;
+  const int text = __ldg(p.text_len + b);
+  const int t0 = p.sys_len + Nv + text;
+  const long long lbh_in = ((long long)l_rel * B + b) * H + h;
+  const long long lbh = ((long long)l * B + b) * H + h;
+  const uint4* srcK = reinterpret_cast<const uint4*>(k + lbh_in * t0_max * D);
+  const uint4* srcV = reinterpret_cast<const uint4*>(v + lbh_in * t0_max * D);
+  T* blk = reinterpret_cast<T*>(p.cache) + lbh * p.lbh_stride;
+  uint4* dKv = reinterpret_cast<uint4*>(blk);
+  uint4* dVv = reinterpret_cast<uint4*>(blk + (long long)Nv * D);
+  uint4* dKt = reinterpret_cast<uint4*>(blk + 2LL * Nv * D);
+  uint4* dVt = reinterpret_cast<uint4*>(blk + 2LL * Nv * D + (long long)p.cap_txt * D);
+  const int total = t0 * VPR;
+  for (int i = blockIdx.x * kThreads + threadIdx.x; i < total; i += gridDim.x * kThreads) {
+    const int row = i / VPR, c = i % VPR;
+    const uint4 kk = __ldg(srcK + i), vv = __ldg(srcV + i);
+    if (row >= p.sys_len && row < p.sys_len + Nv) {
+      const int d = (row - p.sys_len) * VPR + c;
+      dKv[d] = kk; dVv[d] = vv;
+    } else {
+      const int d = (row < p.sys_len ? row : row - Nv) * VPR + c;
+      dKt[d] = kk; dVt[d] = vv;
+    }
+  }
+  if (h == 0 && blockIdx.x == 0) {
+    const long long lb = (long long)l * B + b;
+    for (int i = threadIdx.x; i < Nv; i += kThreads) { p.ids[lb * Nv + i] = i; p.mass_by_id[lb * Nv + i] = 0.f; }
+    if (threadIdx.x == 0) p.n_cur[lb] = Nv;
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+struct Layout {
+  size_t elem, cache, part_ml, part_acc, logits, mass, ids, n_cur, text_len, status, stage_q, stage_k, stage_v,
+      stage_o, total;
+  long long lbh_stride;
+  int cap_txt, chunk_rows, max_items;
+};
+
+bool valid_config(const st3_config* c) {
+  if (!c) return false;
+  if (c->num_layers < 1 || c->num_layers > kMaxLayers) return false;
+  if (c->num_heads < 1 || c->num_heads > kMaxHeads) return false;
+  if (c->head_dim != 64 && c->head_dim != 128) return false;
+  if (c->dtype != ST3_F32 && c->dtype != ST3_BF16) return false;
+  if (c->batch < 1 || c->batch > 4096 || c->sys_len < 0 || c->num_visual < 0 || c->num_visual > kMaxVisual)
+    return false;
+  if (c->max_text_len < 1 || c->max_decode_steps < 0) return false;
+  if (c->first_prune_layer < 0 || c->stride < 1) return false;
+  if (c->first_ratio_bp < 0 || c->first_ratio_bp > 10000 || c->step_ratio_bp < 0 || c->step_ratio_bp > 10000)
+    return false;
+  if (c->anneal < ST3_ANNEAL_COSINE || c->anneal > ST3_ANNEAL_EXP) return false;
+  if ((c->anneal == ST3_ANNEAL_COSINE || c->anneal == ST3_ANNEAL_LINEAR) && !(c->tau > 0.0)) return false;
+  if (c->anneal == ST3_ANNEAL_EXP && !(c->sigma > 0.0)) return false;
+  if (c->rows_per_chunk < 0 || c->rows_per_chunk > kMaxChunkRows) return false;
+  return true;
+}
+
+int pick_chunk_rows(const st3_config* c) {
+  if (c->rows_per_chunk > 0) return c->rows_per_chunk;
+  return 128;
+}
+
+Layout make_layout(const st3_config* c) {
+  Layout L{};
+  L.elem = c->dtype == ST3_BF16 ? 2 : 4;
+  L.cap_txt = c->sys_len + c->max_text_len + c->max_decode_steps;
+  L.chunk_rows = pick_chunk_rows(c);
+  L.lbh_stride = 2LL * ((long long)c->num_visual + L.cap_txt) * c->head_dim;
+  const size_t lb = (size_t)c->num_layers * c->batch;
+  const size_t lbh = lb * c->num_heads;
+  L.max_items = (int)(lb * (ceil_div(c->num_visual, L.chunk_rows) + ceil_div(L.cap_txt, L.chunk_rows)));
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  L.cache = take(lbh * (size_t)L.lbh_stride * L.elem);
+  L.part_ml = take((size_t)L.max_items * c->num_heads * 2 * sizeof(float));
+  L.part_acc = take((size_t)L.max_items * c->num_heads * c->head_dim * sizeof(float));
+  L.logits = take(lbh * (size_t)c->num_visual * sizeof(float));
+  L.mass = take(lb * (size_t)c->num_visual * sizeof(float));
+  L.ids = take(lb * (size_t)c->num_visual * sizeof(int));
+  L.n_cur = take(lb * sizeof(int));
+  L.text_len = take((size_t)c->batch * sizeof(int));
+  L.status = take(256);
+  const size_t io = lbh * c->head_dim * L.elem;
+  L.stage_q = take(io); L.stage_k = take(io); L.stage_v = take(io); L.stage_o = take(io);
+  L.total = off;
+  return L;
+}
+
+double beta_of(const st3_config* c, int t) {
+  if (c->anneal == ST3_ANNEAL_NONE || c->disable_trim) return 1.0;
+  if (c->anneal == ST3_ANNEAL_EXP) return exp(-(double)t / c->sigma);
+  if ((double)t >= c->tau) return 0.0;
+  if (c->anneal == ST3_ANNEAL_COSINE) return cos((double)t * M_PI / (2.0 * c->tau));
+  return 1.0 - (double)t / c->tau;
+}
+
+int count_of(const st3_config* c, int layer, int step) {
+  long long keep_bp = 10000;
+  if (!c->disable_trim && layer >= c->first_prune_layer) {
+    const long long k = (layer - c->first_prune_layer) / c->stride;
+    keep_bp = 10000 - c->first_ratio_bp - k * (long long)c->step_ratio_bp;
+    if (keep_bp < 0) keep_bp = 0;
+  }
+  const long long n0 = (long long)c->num_visual * keep_bp / 10000;
+  if (layer < c->first_prune_layer || step == 0) return (int)n0;
+  return (int)floor((double)n0 * beta_of(c, step) + 1e-9);
+}
+
+}  // namespace
+
+struct st3_ctx {
+  st3_config cfg;
+  Layout lay;
+  unsigned char* ws;
+  std::vector<int> n_tab;      // [L][max_decode_steps + 1]
+  std::vector<int> n_host;     // visual rows each layer holds now (all sequences alike)
+  std::vector<int> last_step;  // -1: not prefilled
+  std::vector<int> text_len;   // host copy
+  bool have_text;
+  int max_text;
+  cudaStream_t last_stream;
+  int64_t launches;
+  bool profiling;
+  std::vector<cudaEvent_t> ev_pool;  // triples: before attend, after attend, after finish
+  size_t ev_used;
+  int attend_smem, finish_smem;
+};
+
+namespace {
+
+template <typename T, int D>
+st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cudaStream_t st, const void* pk,
+                         const void* pv, bool ingest) {
+  const st3_config& c = ctx->cfg;
+  if (ingest) {
+    dim3 grid(8, (unsigned)(c.num_heads * c.batch * p.layer_count));
+    st3_ingest_kernel<T, D><<<grid, kThreads, 0, st>>>(p, reinterpret_cast<const T*>(pk),
+                                                       reinterpret_cast<const T*>(pv),
+                                                       c.sys_len + c.num_visual + c.max_text_len);
+    ctx->launches++;
+  }
+  cudaEvent_t e0 = nullptr, e1 = nullptr, e2 = nullptr;
+  if (ctx->profiling) {
+    while (ctx->ev_pool.size() < ctx->ev_used + 3) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return ST3_ERR_CUDA;
+      ctx->ev_pool.push_back(e);
+    }
+    e0 = ctx->ev_pool[ctx->ev_used]; e1 = ctx->ev_pool[ctx->ev_used + 1]; e2 = ctx->ev_pool[ctx->ev_used + 2];
+    ctx->ev_used += 3;
+    cudaEventRecord(e0, st);
+  }
+  st3_attend_kernel<T, D><<<(unsigned)(total_items * c.num_heads), kThreads, ctx->attend_smem, st>>>(p);
+  if (e1) cudaEventRecord(e1, st);
+  st3_finish_kernel<T, D><<<(unsigned)(p.layer_count * c.batch), kThreads, ctx->finish_smem, st>>>(p);
+  if (e2) cudaEventRecord(e2, st);
+  ctx->launches += 2;
+  return cudaGetLastError() == cudaSuccess ? ST3_OK : ST3_ERR_CUDA;
+}
+
+template <typename T, int D>
+st3_status set_attrs_t(st3_ctx* ctx) {
+  if (cudaFuncSetAttribute(st3_attend_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           ctx->attend_smem) != cudaSuccess)
+    return ST3_ERR_CUDA;
+  if (cudaFuncSetAttribute(st3_finish_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           ctx->finish_smem) != cudaSuccess)
+    return ST3_ERR_CUDA;
+  return ST3_OK;
+}
+
+#define ST3_DISPATCH(ctx, CALL)                                                            \
+  ((ctx)->cfg.dtype == ST3_BF16                                                            \
+       ? ((ctx)->cfg.head_dim == 128 ? CALL(__nv_bfloat16, 128) : CALL(__nv_bfloat16, 64)) \
+       : ((ctx)->cfg.head_dim == 128 ? CALL(float, 128) : CALL(float, 64)))
+
+bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Common body of prefill (step 0, ingest, no append) and decode (step >= 1, append).
+st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, const void* q, const void* k,
+                    const void* v, void* out, cudaStream_t st, bool prefill) {
+  const st3_config& c = ctx->cfg;
+  const Layout& L = ctx->lay;
+  StepParams p;
+  memset(&p, 0, sizeof(p));
+  p.q = q; p.k_new = prefill ? nullptr : k; p.v_new = prefill ? nullptr : v; p.out = out;
+  p.cache = ctx->ws + L.cache;
+  p.part_ml = reinterpret_cast<float*>(ctx->ws + L.part_ml);
+  p.part_acc = reinterpret_cast<float*>(ctx->ws + L.part_acc);
+  p.logits = reinterpret_cast<float*>(ctx->ws + L.logits);
+  p.mass_by_id = reinterpret_cast<float*>(ctx->ws + L.mass);
+  p.ids = reinterpret_cast<int*>(ctx->ws + L.ids);
+  p.n_cur = reinterpret_cast<int*>(ctx->ws + L.n_cur);
+  p.text_len = reinterpret_cast<const int*>(ctx->ws + L.text_len);
+  p.status = reinterpret_cast<int*>(ctx->ws + L.status);
+  p.lbh_stride = L.lbh_stride;
+  p.layer_begin = layer_begin; p.layer_count = layer_count; p.B = c.batch; p.H = c.num_heads;
+  p.sys_len = c.sys_len; p.Nv = c.num_visual; p.cap_txt = L.cap_txt; p.step = step; p.append = prefill ? 0 : 1;
+  p.chunk_rows = L.chunk_rows;
+  const int R = L.chunk_rows;
+  p.ct = ceil_div(c.sys_len + ctx->max_text + step, R);
+  p.cvp[0] = 0;
+  for (int i = 0; i < layer_count; ++i) {
+    const int l = layer_begin + i;
+    const int ncur = prefill ? c.num_visual : ctx->n_host[l];
+    const int tgt = ctx->n_tab[(size_t)l * (c.max_decode_steps + 1) + step];
+    p.ncur[i] = ncur;
+    p.ntgt[i] = tgt < ncur ? tgt : ncur;
+    p.cvp[i + 1] = p.cvp[i] + ceil_div(ncur, R);
+  }
+  const long long total_items = (long long)c.batch * (p.cvp[layer_count] + (long long)layer_count * p.ct);
+  if (total_items > L.max_items || total_items * c.num_heads > 0x7fffffffLL) return ST3_ERR_CAPACITY;
+
+#define ST3_LAUNCH(T, D) launch_step_t<T, D>(ctx, p, (int)total_items, st, k, v, prefill)
+  const st3_status s = ST3_DISPATCH(ctx, ST3_LAUNCH);
+#undef ST3_LAUNCH
+  if (s != ST3_OK) return s;
+  for (int i = 0; i < layer_count; ++i) {
+    ctx->n_host[layer_begin + i] = p.ntgt[i];
+    ctx->last_step[layer_begin + i] = step;
+  }
+  ctx->last_stream = st;
+  return ST3_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------
+// C ABI
+// ------------------------------------------------------------------------------------------
+extern "C" {
+
+int32_t st3_schedule_count(const st3_config* cfg, int32_t layer, int32_t step) {
+  if (!valid_config(cfg) || layer < 0 || layer >= cfg->num_layers || step < 0) return -1;
+  return count_of(cfg, layer, step);
+}
+
+st3_status st3_workspace_size(const st3_config* cfg, size_t* bytes) {
+  if (!valid_config(cfg) || !bytes) return ST3_ERR_INVALID_ARG;
+  *bytes = make_layout(cfg).total;
+  return ST3_OK;
+}
+
+st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, st3_ctx** out) {
+  if (out) *out = nullptr;
+  if (!valid_config(cfg) || !out || !dev_workspace) return ST3_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(dev_workspace) & 255u) return ST3_ERR_INVALID_ARG;
+  const Layout L = make_layout(cfg);
+  if (bytes < L.total) return ST3_ERR_WORKSPACE_TOO_SMALL;
+  st3_ctx* ctx = new (std::nothrow) st3_ctx();
+  if (!ctx) return ST3_ERR_INVALID_ARG;
+  ctx->cfg = *cfg;
+  ctx->lay = L;
+  ctx->ws = static_cast<unsigned char*>(dev_workspace);
+  const int T = cfg->max_decode_steps + 1;
+  ctx->n_tab.resize((size_t)cfg->num_layers * T);
+  for (int l = 0; l < cfg->num_layers; ++l)
+    for (int t = 0; t < T; ++t) ctx->n_tab[(size_t)l * T + t] = count_of(cfg, l, t);
+  ctx->n_host.assign(cfg->num_layers, cfg->num_visual);
+  ctx->last_step.assign(cfg->num_layers, -1);
+  ctx->text_len.assign(cfg->batch, 0);
+  ctx->have_text = false;
+  ctx->max_text = 0;
+  ctx->last_stream = nullptr;
+  ctx->launches = 0;
+  ctx->profiling = false;
+  ctx->ev_used = 0;
+  const size_t rowb = (size_t)cfg->head_dim * L.elem;
+  ctx->attend_smem = (int)(2 * (size_t)L.chunk_rows * rowb + (size_t)L.chunk_rows * sizeof(float));
+  ctx->finish_smem = (int)((size_t)cfg->num_visual * 16 + 16);
+  if (ctx->attend_smem > 200 * 1024 || ctx->finish_smem > 200 * 1024) { delete ctx; return ST3_ERR_UNSUPPORTED; }
+#define ST3_ATTR(T, D) set_attrs_t<T, D>(ctx)
+  st3_status s = ST3_DISPATCH(ctx, ST3_ATTR);
+#undef ST3_ATTR
+  if (s == ST3_OK) {
+    // bookkeeping area (scores, ids, counts, text lengths, status word) starts cleared
+    if (cudaMemsetAsync(ctx->ws + L.mass, 0, L.stage_q - L.mass, nullptr) != cudaSuccess ||
+        cudaStreamSynchronize(nullptr) != cudaSuccess)
+      s = ST3_ERR_CUDA;
+  }
+  if (s != ST3_OK) { delete ctx; return s; }
+  *out = ctx;
+  return ST3_OK;
+}
+
+st3_status st3_prefill_select(st3_ctx* ctx, int32_t layer_begin, int32_t layer_count, const void* q_last,
+                              const void* k, const void* v, const int32_t* text_len, void* out,
+                              void* cuda_stream) {
+  if (!ctx || !text_len) return ST3_ERR_INVALID_ARG;
+  const st3_config& c = ctx->cfg;
+  if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c.num_layers) return ST3_ERR_INVALID_ARG;
+  if (!aligned16(q_last) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return ST3_ERR_INVALID_ARG;
+  int mx = 0;
+  for (int b = 0; b < c.batch; ++b) {
+    if (text_len[b] < 1) return ST3_ERR_INVALID_ARG;
+    if (text_len[b] > c.max_text_len) return ST3_ERR_CAPACITY;
+    mx = text_len[b] > mx ? text_len[b] : mx;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  bool changed = !ctx->have_text;
+  for (int b = 0; b < c.batch && !changed; ++b) changed = ctx->text_len[b] != text_len[b];
+  if (changed) {
+    // a new generation: every layer must be prefilled again before it can decode
+    for (int b = 0; b < c.batch; ++b) ctx->text_len[b] = text_len[b];
+    ctx->max_text = mx;
+    ctx->have_text = true;
+    for (int l = 0; l < c.num_layers; ++l) ctx->last_step[l] = -1;
+    // pageable source: the runtime stages it before returning, so ctx->text_len may change later
+    if (cudaMemcpyAsync(ctx->ws + ctx->lay.text_len, ctx->text_len.data(), (size_t)c.batch * sizeof(int),
+                        cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return ST3_ERR_CUDA;
+  }
+  return run_step(ctx, 0, layer_begin, layer_count, q_last, k, v, out, st, true);
+}
+
+st3_status st3_decode_step(st3_ctx* ctx, int32_t step, int32_t layer_begin, int32_t layer_count, const void* q,
+                           const void* k_new, const void* v_new, void* out, void* cuda_stream) {
+  if (!ctx) return ST3_ERR_INVALID_ARG;
+  const st3_config& c = ctx->cfg;
+  if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c.num_layers) return ST3_ERR_INVALID_ARG;
+  if (step < 1) return ST3_ERR_INVALID_ARG;
+  if (step > c.max_decode_steps) return ST3_ERR_CAPACITY;
+  if (!aligned16(q) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return ST3_ERR_INVALID_ARG;
+  if (!ctx->have_text) return ST3_ERR_BAD_STATE;
+  for (int l = layer_begin; l < layer_begin + layer_count; ++l)
+    if (ctx->last_step[l] != step - 1) return ST3_ERR_BAD_STATE;
+  return run_step(ctx, step, layer_begin, layer_count, q, k_new, v_new, out, static_cast<cudaStream_t>(cuda_stream),
+                  false);
+}
+
+st3_status st3_decode_step_host(st3_ctx* ctx, int32_t step, int32_t layer_begin, int32_t layer_count,
+                                const void* q_host, const void* k_new_host, const void* v_new_host, void* out_host,
+                                void* cuda_stream) {
+  if (!ctx || !q_host || !k_new_host || !v_new_host || !out_host) return ST3_ERR_INVALID_ARG;
+  const st3_config& c = ctx->cfg;
+  if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c.num_layers) return ST3_ERR_INVALID_ARG;
+  const Layout& L = ctx->lay;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t bytes = (size_t)layer_count * c.batch * c.num_heads * c.head_dim * L.elem;
+  unsigned char* dq = ctx->ws + L.stage_q; unsigned char* dk = ctx->ws + L.stage_k;
+  unsigned char* dv = ctx->ws + L.stage_v; unsigned char* dout = ctx->ws + L.stage_o;
+  if (cudaMemcpyAsync(dq, q_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(dk, k_new_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpyAsync(dv, v_new_host, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return ST3_ERR_CUDA;
+  const st3_status s = st3_decode_step(ctx, step, layer_begin, layer_count, dq, dk, dv, dout, cuda_stream);
+  if (s != ST3_OK) return s;
+  if (cudaMemcpyAsync(out_host, dout, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ST3_ERR_CUDA;
+  return ST3_OK;
+}
+
+st3_status st3_get_kept(st3_ctx* ctx, int32_t layer, int32_t* ids, int32_t* count, float* mass, void* cuda_stream) {
+  if (!ctx || !ids || !count) return ST3_ERR_INVALID_ARG;
+  const st3_config& c = ctx->cfg;
+  if (layer < 0 || layer >= c.num_layers) return ST3_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const Layout& L = ctx->lay;
+  const size_t per = (size_t)c.batch * c.num_visual;
+  if (per && cudaMemcpyAsync(ids, ctx->ws + L.ids + layer * per * sizeof(int), per * sizeof(int),
+                             cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return ST3_ERR_CUDA;
+  if (cudaMemcpyAsync(count, ctx->ws + L.n_cur + (size_t)layer * c.batch * sizeof(int), (size_t)c.batch * sizeof(int),
+                      cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return ST3_ERR_CUDA;
+  if (mass && per && cudaMemcpyAsync(mass, ctx->ws + L.mass + layer * per * sizeof(float), per * sizeof(float),
+                                     cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+    return ST3_ERR_CUDA;
+  ctx->last_stream = st;
+  return ST3_OK;
+}
+
+st3_status st3_get_rows(st3_ctx* ctx, int32_t layer, int32_t b, int32_t h, void* k_vis, void* v_vis, void* k_txt,
+                        void* v_txt, void* cuda_stream) {
+  if (!ctx) return ST3_ERR_INVALID_ARG;
+  const st3_config& c = ctx->cfg;
+  if (layer < 0 || layer >= c.num_layers || b < 0 || b >= c.batch || h < 0 || h >= c.num_heads)
+    return ST3_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const Layout& L = ctx->lay;
+  const size_t rowb = (size_t)c.head_dim * L.elem;
+  const unsigned char* blk =
+      ctx->ws + L.cache + (((size_t)layer * c.batch + b) * c.num_heads + h) * (size_t)L.lbh_stride * L.elem;
+  const size_t nv = (size_t)c.num_visual * rowb, nt = (size_t)L.cap_txt * rowb;
+  void* dst[4] = {k_vis, v_vis, k_txt, v_txt};
+  const size_t off[4] = {0, nv, 2 * nv, 2 * nv + nt};
+  const size_t len[4] = {nv, nv, nt, nt};
+  for (int i = 0; i < 4; ++i)
+    if (dst[i] && len[i] &&
+        cudaMemcpyAsync(dst[i], blk + off[i], len[i], cudaMemcpyDeviceToDevice, st) != cudaSuccess)
+      return ST3_ERR_CUDA;
+  ctx->last_stream = st;
+  return ST3_OK;
+}
+
+st3_status st3_get_status(st3_ctx* ctx, int32_t* word) {
+  if (!ctx || !word) return ST3_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(ctx->last_stream) != cudaSuccess) return ST3_ERR_CUDA;
+  int w = 0;
+  if (cudaMemcpy(&w, ctx->ws + ctx->lay.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return ST3_ERR_CUDA;
+  *word = w;
+  return w ? ST3_ERR_DEVICE_CHECK : ST3_OK;
+}
+
+st3_status st3_rows_held(st3_ctx* ctx, int64_t* visual_rows, int64_t* other_rows) {
+  if (!ctx) return ST3_ERR_INVALID_ARG;
+  const st3_config& c = ctx->cfg;
+  int64_t vis = 0, oth = 0;
+  for (int l = 0; l < c.num_layers; ++l) {
+    if (ctx->last_step[l] < 0) continue;
+    vis += (int64_t)ctx->n_host[l] * c.batch;
+    for (int b = 0; b < c.batch; ++b) oth += c.sys_len + ctx->text_len[b] + ctx->last_step[l];
+  }
+  if (visual_rows) *visual_rows = vis;
+  if (other_rows) *other_rows = oth;
+  return ST3_OK;
+}
+
+st3_status st3_profile_enable(st3_ctx* ctx, int32_t on) {
+  if (!ctx) return ST3_ERR_INVALID_ARG;
+  ctx->profiling = on != 0;
+  ctx->ev_used = 0;
+  return ST3_OK;
+}
+
+st3_status st3_profile_read(st3_ctx* ctx, double* attn_ms, double* finish_ms, int64_t* attn_launches,
+                            int64_t* finish_launches) {
+  if (!ctx) return ST3_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(ctx->last_stream) != cudaSuccess) return ST3_ERR_CUDA;
+  double a = 0, f = 0;
+  int64_t n = 0;
+  for (size_t i = 0; i + 3 <= ctx->ev_used; i += 3) {
+    float ms = 0;
+    if (cudaEventElapsedTime(&ms, ctx->ev_pool[i], ctx->ev_pool[i + 1]) != cudaSuccess) return ST3_ERR_CUDA;
+    a += ms;
+    if (cudaEventElapsedTime(&ms, ctx->ev_pool[i + 1], ctx->ev_pool[i + 2]) != cudaSuccess) return ST3_ERR_CUDA;
+    f += ms;
+    ++n;
+  }
+  ctx->ev_used = 0;
+  if (attn_ms) *attn_ms = a;
+  if (finish_ms) *finish_ms = f;
+  if (attn_launches) *attn_launches = n;
+  if (finish_launches) *finish_launches = n;
+  return ST3_OK;
+}
+
+int64_t st3_launch_count(const st3_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* st3_status_string(st3_status s) {
+  switch (s) {
+    case ST3_OK: return "ok";
+    case ST3_ERR_INVALID_ARG: return "invalid argument";
+    case ST3_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case ST3_ERR_BAD_STATE: return "call order violated";
+    case ST3_ERR_CAPACITY: return "capacity exceeded";
+    case ST3_ERR_CUDA: return "CUDA runtime error";
+    case ST3_ERR_DEVICE_CHECK: return "device-side check failed";
+    case ST3_ERR_UNSUPPORTED: return "unsupported shape";
+  }
+  return "unknown status";
+}
+
+st3_status st3_destroy(st3_ctx* ctx) {
+  if (!ctx) return ST3_ERR_INVALID_ARG;
+  for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+  delete ctx;
+  return ST3_OK;
+}
+
+}  // extern "C"

@@ -365,7 +365,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p) {
   constexpr int ROWB = D * sizeof(T);
   constexpr int VPR = ROWB / 16;  // 16-byte vectors per row
-  extern __shared__ __align__(16) unsigned char smem[];
+  extern __shared__ __align__(128) unsigned char smem[];
   __shared__ float s_M[kMaxHeads];
   __shared__ float s_invL[kMaxHeads];
   __shared__ int s_hist[256];

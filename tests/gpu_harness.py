@@ -1,0 +1,164 @@
+"""Drives the CUDA path through the C ABI on a synthetic workload and checks it against the oracle.
+
+Parity is teacher-forced: before judging a step the oracle's cache for a (sequence, layer) unit is
+rebuilt from the kept ids the GPU holds, so every step is compared on identical state; the kept
+set after the step is judged with the near-tie acceptance rule.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from oracle import st3_oracle as O
+from paper_2412_20105_b200 import binding as B
+from synth import SynthInputs, Workload
+from helpers import make_schedule, rebuild_cache, check_kept, f64
+
+OUT_ABS_F32 = 2e-3          # max-abs bound for fp32 outputs
+OUT_REL_BF16 = 2e-2         # relative bound for bf16 outputs ...
+OUT_FLOOR_BF16 = 1e-2       # ... relative to max(|ref|, this floor)
+MASS_RTOL, MASS_ATOL = 5e-4, 1e-9
+
+
+def assert_out_close(got: np.ndarray, ref: np.ndarray, dtype: str, where=""):
+    assert np.all(np.isfinite(got)), where
+    if dtype == "f32":
+        err = np.abs(got - ref).max()
+        assert err <= OUT_ABS_F32, f"{where}: max-abs {err}"
+    else:
+        rel = np.abs(got - ref) / np.maximum(np.abs(ref), OUT_FLOOR_BF16)
+        assert rel.max() <= OUT_REL_BF16, f"{where}: max-rel {rel.max()}"
+
+
+class GpuRun:
+    def __init__(self, wl: Workload, device="cuda:0", **cfg_overrides):
+        self.wl, self.dev = wl, torch.device(device)
+        self.g = SynthInputs(wl)
+        self.sched = make_schedule(wl, disable_trim=bool(cfg_overrides.get("disable_trim", 0)))
+        self.cfg = B.config_from_workload(wl, **cfg_overrides)
+        self.ctx = B.Context(self.cfg, device)
+        self.L = wl.num_layers
+        self.out = torch.empty(self.ctx.io_shape(), dtype=self.ctx.dtype, device=self.dev)
+        self.stats = {"exact": 0, "near-tie": 0, "units": 0}
+
+    def close(self):
+        self.ctx.close()
+
+    # ------------------------------------------------------------------ running
+    def prefill(self, layers_per_call=None):
+        wl, g = self.wl, self.g
+        step = layers_per_call or self.L
+        q0 = g.queries([0], device=self.dev)[0]
+        for l0 in range(0, self.L, step):
+            ls = list(range(l0, min(self.L, l0 + step)))
+            K, V = g.prompt_kv(ls, device=self.dev)
+            self.ctx.prefill_select(q0[l0:l0 + len(ls)].contiguous(), K, V, g.text_len.tolist(),
+                                    self.out[l0:l0 + len(ls)], layer_begin=l0)
+            del K, V
+        self.q_cur = q0
+        return self.out
+
+    def inputs(self, step):
+        g = self.g
+        q = g.queries([step], device=self.dev)[0]
+        kn, vn = g.new_kv([step], device=self.dev)
+        return q, kn[0], vn[0]
+
+    def decode(self, step, layers_per_call=None):
+        q, kn, vn = self.inputs(step)
+        lpc = layers_per_call or self.L
+        for l0 in range(0, self.L, lpc):
+            n = min(lpc, self.L - l0)
+            self.ctx.decode_step(step, q[l0:l0 + n], kn[l0:l0 + n], vn[l0:l0 + n], self.out[l0:l0 + n],
+                                 layer_begin=l0)
+        self.q_cur, self.kn_cur, self.vn_cur = q, kn, vn
+        return self.out
+
+    def kept(self, layer):
+        ids, cnt, mass = self.ctx.get_kept(layer)
+        return ids.cpu().numpy(), cnt.cpu().numpy(), mass.cpu().numpy()
+
+    def snapshot(self, layers):
+        """{layer: (ids [B, Nv], count [B])} of the current device state."""
+        return {l: self.kept(l)[:2] for l in layers}
+
+    # ------------------------------------------------------------------ checking
+    def check_prefill_unit(self, b, l):
+        wl, g, s = self.wl, self.g, self.sched
+        t0 = wl.sys_len + wl.num_visual + int(g.text_len[b])
+        K, V = g.kv_rows([b], [l], range(t0))
+        q = g.queries([0], [l])[0, 0, b]
+        ref_out, ref_mass, _ = O.prefill_select(f64(q), f64(K[0, 0]), f64(V[0, 0]), wl.sys_len, wl.num_visual,
+                                                s.n0(l))
+        got = f64(self.out[l, b])
+        assert_out_close(got, ref_out, wl.dtype, f"prefill out b={b} l={l}")
+        ids, cnt, mass = self.kept(l)
+        n = int(cnt[b])
+        assert n == s.n0(l), (n, s.n0(l))
+        self._judge(ref_mass, np.arange(wl.num_visual), s.n0(l), ids[b, :n], mass[b], trimmed=s.n0(l) < wl.num_visual,
+                    where=f"prefill b={b} l={l}")
+
+    def check_decode_unit(self, b, l, step, before):
+        """`before` = (ids [B, Nv], count [B]) of layer l taken before the step ran."""
+        wl, g, s = self.wl, self.g, self.sched
+        ids_b, cnt_b = before
+        nb = int(cnt_b[b])
+        cache = rebuild_cache(wl, g, b, l, ids_b[b, :nb], step - 1)
+        ref_out, ref_mass, ids_before = O.decode_step(cache, f64(self.q_cur[l, b]), f64(self.kn_cur[l, b]),
+                                                      f64(self.vn_cur[l, b]), s.n(l, step))
+        assert_out_close(f64(self.out[l, b]), ref_out, wl.dtype, f"decode out b={b} l={l} t={step}")
+        ids, cnt, mass = self.kept(l)
+        n = int(cnt[b])
+        assert n == s.n(l, step) == min(nb, s.n(l, step)), (n, s.n(l, step), nb)
+        self._judge(ref_mass, ids_before, n, ids[b, :n], mass[b], trimmed=n < nb, where=f"decode b={b} l={l} t={step}")
+
+    def _judge(self, ref_mass, ids_before, k, got_ids, got_mass_by_id, trimmed, where):
+        assert len(set(got_ids.tolist())) == len(got_ids), f"{where}: duplicate ids"
+        if trimmed:
+            gm = got_mass_by_id[np.asarray(ids_before, dtype=np.int64)]
+            assert np.allclose(gm, ref_mass, rtol=MASS_RTOL, atol=MASS_ATOL), \
+                f"{where}: mass max rel err {np.max(np.abs(gm - ref_mass) / np.maximum(ref_mass, 1e-12))}"
+        verdict = check_kept(ref_mass, np.asarray(ids_before), k, got_ids)
+        self.stats[verdict] += 1
+        self.stats["units"] += 1
+
+    def check_rows_unit(self, b, l, h, step):
+        """Cache rows are bit-identical to the generated rows their ids name; text rows are [S | I | O]."""
+        wl, g = self.wl, self.g
+        ids, cnt, _ = self.kept(l)
+        n = int(cnt[b])
+        kv, vv, kt, vt = self.ctx.get_rows(l, b, h)
+        text = int(g.text_len[b])
+        if n:
+            Kr, Vr = g.kv_rows([b], [l], (wl.sys_len + ids[b, :n]).tolist())
+            assert torch.equal(kv[:n].cpu(), Kr[0, 0, h]) and torch.equal(vv[:n].cpu(), Vr[0, 0, h])
+        toks = list(range(wl.sys_len)) + list(range(wl.sys_len + wl.num_visual, wl.sys_len + wl.num_visual + text)) \
+            + [g.gen_token(s) for s in range(1, step + 1)]
+        Kt, Vt = g.kv_rows([b], [l], toks)
+        assert torch.equal(kt[:len(toks)].cpu(), Kt[0, 0, h]) and torch.equal(vt[:len(toks)].cpu(), Vt[0, 0, h])
+
+
+def run_and_check(wl: Workload, steps, check_steps=None, units=None, layers_per_call=None, rows_checks=2, **cfg):
+    """Prefill + decode `steps` steps; check every (b, l) unit (or the sampled `units`) at `check_steps`."""
+    run = GpuRun(wl, **cfg)
+    try:
+        all_units = [(b, l) for l in range(wl.num_layers) for b in range(wl.batch)]
+        units = all_units if units is None else units
+        check_steps = set(range(0, steps + 1)) if check_steps is None else set(check_steps)
+        layers = sorted(set(l for _, l in units))
+        run.prefill(layers_per_call)
+        if 0 in check_steps:
+            for b, l in units:
+                run.check_prefill_unit(b, l)
+        for t in range(1, steps + 1):
+            before = run.snapshot(layers) if t in check_steps else None
+            run.decode(t, layers_per_call)
+            if t in check_steps:
+                for b, l in units:
+                    run.check_decode_unit(b, l, t, before[l])
+                for b, l in units[:rows_checks]:
+                    run.check_rows_unit(b, l, (t * 7) % wl.num_heads, t)
+        assert run.ctx.status() == 0
+        return run.stats
+    finally:
+        run.close()

@@ -1,0 +1,82 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 oracle on the synthetic workloads."""
+import numpy as np
+import pytest
+import torch
+
+from synth import SynthInputs, get_workload
+from gpu_harness import run_and_check, GpuRun
+
+pytestmark = pytest.mark.gpu
+
+
+def test_generator_is_bit_identical_on_cpu_and_gpu():
+    wl = get_workload("llava15_7b")
+    g = SynthInputs(wl)
+    Kc, Vc = g.kv_rows([0], [7], range(0, wl.t0_max, 3))
+    Kg, Vg = g.kv_rows([0], [7], range(0, wl.t0_max, 3), device="cuda:0")
+    assert torch.equal(Kc, Kg.cpu()) and torch.equal(Vc, Vg.cpu())
+    assert torch.equal(g.queries([0, 5], [7]), g.queries([0, 5], [7], device="cuda:0").cpu())
+
+
+@pytest.mark.parametrize("tau", [50.0, 10.0])
+def test_tiny_every_step(tau):
+    wl = get_workload("tiny").scaled(tau=tau)
+    stats = run_and_check(wl, wl.decode_steps)
+    assert stats["units"] == wl.decode_steps + 1
+
+
+@pytest.mark.parametrize("rows", [16, 64, 100, 256])
+def test_tiny_chunk_sizes_and_ragged_tails(rows):
+    wl = get_workload("tiny")
+    run_and_check(wl, 6, rows_per_chunk=rows)
+
+
+def test_tiny_untrimmed_equals_full_attention():
+    wl = get_workload("tiny")
+    stats = run_and_check(wl, 4, disable_trim=1)
+    assert stats["near-tie"] == 0
+
+
+@pytest.mark.parametrize("dtype,D,H", [("f32", 128, 3), ("bf16", 64, 5), ("bf16", 128, 2), ("f32", 64, 1)])
+def test_small_odd_shapes(dtype, D, H):
+    wl = get_workload("tiny").scaled(dtype=dtype, head_dim=D, num_heads=H, num_layers=5, batch=3, sys_len=3,
+                                     num_visual=131, text_len_min=1, text_len_max=37, decode_steps=9,
+                                     first_prune_layer=1, stride=2, step_ratio_bp=2000, tau=9.0, num_planted=7)
+    run_and_check(wl, 9)
+    run_and_check(wl, 5, layers_per_call=2)
+
+
+def test_no_visual_tokens_and_single_text_token():
+    wl = get_workload("tiny").scaled(num_visual=0, num_planted=0, sys_len=0, text_len_min=1, text_len_max=1,
+                                     decode_steps=3)
+    run_and_check(wl, 3)
+
+
+def test_llava15_7b_first_steps_all_units():
+    wl = get_workload("llava15_7b")
+    stats = run_and_check(wl, 3)
+    assert stats["units"] == 32 * 4
+
+
+def test_llava15_7b_full_length_sampled_steps():
+    wl = get_workload("llava15_7b")
+    steps = [0, 1, 2, 17, 64, 128, 129, 200, 254, 255, 256]
+    stats = run_and_check(wl, wl.decode_steps, check_steps=steps)
+    assert stats["units"] == 32 * len(steps)
+
+
+def _sampled_units(wl, n, seed):
+    r = np.random.default_rng(seed)
+    layers = [0, 3, wl.num_layers - 1] + r.integers(0, wl.num_layers, size=n).tolist()
+    return [(int(r.integers(wl.batch)), int(l)) for l in layers]
+
+
+@pytest.mark.parametrize("name,steps", [("llava15_7b_b32", [0, 1, 100, 300, 511, 512]),
+                                        ("llava15_13b_b16", [0, 1, 256, 512]),
+                                        ("llava_next_b8", [0, 1, 500, 1023, 1024])])
+def test_full_size_workloads_sampled_units(name, steps):
+    wl = get_workload(name)
+    units = _sampled_units(wl, 5, wl.seed)
+    lpc = 8 if wl.batch > 1 else None
+    stats = run_and_check(wl, wl.decode_steps, check_steps=steps, units=units, layers_per_call=None, rows_checks=1)
+    assert stats["units"] == len(units) * len(steps)

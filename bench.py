@@ -1,0 +1,402 @@
+#!/usr/bin/env python
+"""Benchmark of the ST^3 decode-attention + trimming path on synthetic LLaVA-shaped workloads.
+
+One bench "step" is one whole pass of the hot path over one batch: prefill-select of every layer
+followed by all decode steps of the workload (append, attend, score, select, compact).  The
+metric is decode tokens per second = sequences x decode steps / time.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+Prints ONE JSON line on rank 0.  `--impl reference` times the CPU oracle on a bounded sample of
+the same workload (see `cpu_baseline.sample` in its line).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+for _p in (ROOT, os.path.join(ROOT, "tests")):
+    if _p not in sys.path:
+        sys.path.insert(0, _p)
+
+import numpy as np
+import torch
+
+from synth import SynthInputs, get_workload
+
+METRIC = "decode-step attn+trim tokens/s at LLaVA-1.5-7B shape"
+UNIT = "tokens/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------------------------
+# algorithmic bytes of the attention kernel
+# ----------------------------------------------------------------------------------------------
+def attend_bytes(wl, cfg, B_mod, text_len, step):
+    """Bytes the attention kernel of one launch must move (all layers, all sequences).
+
+    Per (sequence, layer): every cached K and V row once (r*T_cur, the newest row read from the
+    step's inputs), the newest row written to the cache (r), the query (H*D*e) and, where the
+    layer evicts at this step, one fp32 logit per head per visual row (4*H*n_cur).
+    """
+    e = 2 if wl.dtype == "bf16" else 4
+    H, D = wl.num_heads, wl.head_dim
+    r = 2 * H * D * e
+    total = 0
+    for l in range(wl.num_layers):
+        n_cur = wl.num_visual if step == 0 else B_mod.st3_schedule_count(cfg, l, step - 1)
+        n_tgt = B_mod.st3_schedule_count(cfg, l, step)
+        for b in range(wl.batch):
+            t_cur = wl.sys_len + n_cur + int(text_len[b]) + step
+            total += r * t_cur + (r if step > 0 else 0) + H * D * e
+            if n_tgt < n_cur:
+                total += 4 * H * n_cur
+    return total
+
+
+# ----------------------------------------------------------------------------------------------
+# our arm
+# ----------------------------------------------------------------------------------------------
+class Job:
+    """All device-resident inputs of one workload plus a library context."""
+
+    def __init__(self, wl, device, disable_trim=False, rows_per_chunk=0):
+        from paper_2412_20105_b200 import binding as B
+        from paper_2412_20105_b200.build import build
+        build()
+        self.B = B
+        self.wl, self.dev = wl, device
+        self.g = SynthInputs(wl)
+        self.cfg = B.config_from_workload(wl, disable_trim=int(disable_trim), rows_per_chunk=rows_per_chunk)
+        self.ctx = B.Context(self.cfg, device)
+        self.lib = B.load()
+        L, T = wl.num_layers, wl.decode_steps
+        g = self.g
+        self.q0 = g.queries([0], device=device)[0].contiguous()
+        Ks, Vs = [], []
+        for l in range(L):
+            K, V = g.prompt_kv([l], device=device)
+            Ks.append(K); Vs.append(V)
+        self.K, self.V = torch.cat(Ks), torch.cat(Vs)
+        del Ks, Vs
+        chunk = 32
+        qs, ks, vs = [], [], []
+        for s0 in range(1, T + 1, chunk):
+            steps = list(range(s0, min(T, s0 + chunk - 1) + 1))
+            qs.append(g.queries(steps, device=device))
+            kn, vn = g.new_kv(steps, device=device)
+            ks.append(kn); vs.append(vn)
+        self.q, self.kn, self.vn = torch.cat(qs), torch.cat(ks), torch.cat(vs)        # [T, L, B, H, D]
+        self.out = torch.empty_like(self.q)
+        self.out0 = torch.empty_like(self.q0)
+        self.io_bytes = self.q0.numel() * self.q0.element_size()
+        self.text = g.text_len.tolist()
+        self.stream = torch.cuda.current_stream(device).cuda_stream
+
+    def generation(self):
+        """prefill-select + every decode step, device-resident inputs."""
+        B, h, L, st = self.B, self.ctx.handle, self.wl.num_layers, self.stream
+        B.st3_prefill_select(h, 0, L, self.q0.data_ptr(), self.K.data_ptr(), self.V.data_ptr(), self.text,
+                             self.out0.data_ptr(), st)
+        q, k, v, o, nb = self.q.data_ptr(), self.kn.data_ptr(), self.vn.data_ptr(), self.out.data_ptr(), self.io_bytes
+        step_fn = self.lib.st3_decode_step
+        for t in range(1, self.wl.decode_steps + 1):
+            off = (t - 1) * nb
+            rc = step_fn(h, t, 0, L, q + off, k + off, v + off, o + off, st)
+            if rc:
+                raise B.St3Error(rc, f"st3_decode_step t={t}")
+
+    def make_host(self):
+        self.hK, self.hV = self.K.cpu().pin_memory(), self.V.cpu().pin_memory()
+        self.hq0 = self.q0.cpu().pin_memory()
+        self.hq, self.hk, self.hv = self.q.cpu().pin_memory(), self.kn.cpu().pin_memory(), self.vn.cpu().pin_memory()
+        self.hout = torch.empty_like(self.hq).pin_memory()
+        self.hout0 = torch.empty_like(self.hq0).pin_memory()
+        self.dK, self.dV, self.dq0 = torch.empty_like(self.K), torch.empty_like(self.V), torch.empty_like(self.q0)
+
+    def generation_host(self):
+        """Same work, every input starting in pinned host memory and every output ending there."""
+        B, h, L, st = self.B, self.ctx.handle, self.wl.num_layers, self.stream
+        self.dK.copy_(self.hK, non_blocking=True)
+        self.dV.copy_(self.hV, non_blocking=True)
+        self.dq0.copy_(self.hq0, non_blocking=True)
+        B.st3_prefill_select(h, 0, L, self.dq0.data_ptr(), self.dK.data_ptr(), self.dV.data_ptr(), self.text,
+                             self.out0.data_ptr(), st)
+        self.hout0.copy_(self.out0, non_blocking=True)
+        q, k, v, o, nb = self.hq.data_ptr(), self.hk.data_ptr(), self.hv.data_ptr(), self.hout.data_ptr(), self.io_bytes
+        step_fn = self.lib.st3_decode_step_host
+        for t in range(1, self.wl.decode_steps + 1):
+            off = (t - 1) * nb
+            rc = step_fn(h, t, 0, L, q + off, k + off, v + off, o + off, st)
+            if rc:
+                raise B.St3Error(rc, f"st3_decode_step_host t={t}")
+
+    def h2d_bytes(self):
+        kv = 2 * self.K.numel() * self.K.element_size()
+        return kv + self.io_bytes + 3 * self.io_bytes * self.wl.decode_steps
+
+    def d2h_bytes(self):
+        return self.io_bytes * (self.wl.decode_steps + 1)
+
+
+def timed(fn, n, dist):
+    """Device time of n calls of fn in ms (CUDA events on the current stream, max over ranks)."""
+    torch.cuda.synchronize()
+    if dist:
+        torch.distributed.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(n):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    if dist:
+        torch.distributed.barrier()
+    ms = e0.elapsed_time(e1)
+    if dist:
+        t = torch.tensor([ms], device="cuda")
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms
+
+
+def oracle_sample(wl, g, K, V, q0, q, kn, vn, nsteps, warm_steps, reps=1):
+    """Times the oracle, as it stands, on decode steps 1..nsteps of the workload (all layers, all
+    sequences, free-running after its own prefill).  Returns (tokens/s, seconds, threads)."""
+    from oracle import st3_oracle as O
+    from helpers import make_schedule, f64
+    sched = make_schedule(wl)
+    caches = {}
+    for l in range(wl.num_layers):
+        for b in range(wl.batch):
+            t0 = wl.sys_len + wl.num_visual + int(g.text_len[b])
+            _, _, caches[(b, l)] = O.prefill_select(f64(q0[l, b]), f64(K[l, b][:, :t0]), f64(V[l, b][:, :t0]),
+                                                    wl.sys_len, wl.num_visual, sched.n0(l))
+
+    def run(t):
+        for l in range(wl.num_layers):
+            for b in range(wl.batch):
+                O.decode_step(caches[(b, l)], f64(q[t - 1, l, b]), f64(kn[t - 1, l, b]), f64(vn[t - 1, l, b]),
+                              sched.n(l, t))
+
+    t = 1
+    for _ in range(warm_steps):
+        run(t); t += 1
+    t_start = time.perf_counter()
+    first = t
+    for _ in range(nsteps):
+        run(t); t += 1
+    secs = time.perf_counter() - t_start
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = 1
+    return wl.batch * nsteps / secs, secs, threads, first, t - 1
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="llava15_7b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--rows-per-chunk", type=int, default=0)
+    ap.add_argument("--no-extras", action="store_true", help="skip unpruned / cpu_baseline / e2e legs")
+    args = ap.parse_args()
+    wl = get_workload(args.workload)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    config = {"workload": f"{wl.name}: B={wl.batch} L={wl.num_layers} H={wl.num_heads} D={wl.head_dim} "
+                          f"{wl.dtype}, prompt {wl.sys_len}+{wl.num_visual}+[{wl.text_len_min},{wl.text_len_max}], "
+                          f"{wl.decode_steps} decode steps, S={wl.stride} R={wl.step_ratio_bp}bp "
+                          f"P={wl.first_ratio_bp}bp tau={wl.tau:g}",
+              "step": "prefill-select of all layers + all decode steps of one batch",
+              "l2": "inputs larger than L2 (per-step K/V working set > 126 MB); no explicit flush",
+              "parallelism": f"{args.gpus} independent replica(s), no collectives"}
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        g = SynthInputs(wl)
+        s_per = 4 if wl.batch == 1 else 1
+        n_timed, n_warm = args.steps * s_per, max(1, args.warmup) * s_per
+        need = n_timed + n_warm
+        L = wl.num_layers
+        q0 = g.queries([0])[0]
+        K = torch.cat([g.prompt_kv([l])[0] for l in range(L)]) if False else None
+        Ks, Vs = zip(*[g.prompt_kv([l]) for l in range(L)])
+        K, V = torch.cat(Ks), torch.cat(Vs)
+        steps = list(range(1, need + 1))
+        q = g.queries(steps)
+        kn, vn = g.new_kv(steps)
+        val, secs, threads, s_first, s_last = oracle_sample(wl, g, K, V, q0, q, kn, vn, n_timed, n_warm)
+        sample = (f"oracle (numpy fp64), all {L} layers x {wl.batch} sequence(s), decode steps {s_first}-{s_last} of "
+                  f"{wl.decode_steps} after its own prefill; one bench step = {s_per} decode step(s)")
+        line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs * 1e3 / args.steps,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                "data": "synthetic", "config": config,
+                "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+                "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                "gpu_launches": 0}
+        print(json.dumps(line))
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    dist = world > 1
+    torch.cuda.set_device(local)
+    device = torch.device(f"cuda:{local}")
+    if dist:
+        torch.distributed.init_process_group("nccl", device_id=device)
+    if dist:
+        wl = wl.scaled(seed=wl.seed + 1000 * rank)       # replicas work on different data
+    job = Job(wl, device, rows_per_chunk=args.rows_per_chunk)
+    B = job.B
+    tokens_per_gen = wl.batch * wl.decode_steps
+
+    for _ in range(max(3, args.warmup)):
+        job.generation()
+    job.ctx.status()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    n0 = job.ctx.launch_count()
+    ms = timed(job.generation, args.steps, dist)
+    launches = job.ctx.launch_count() - n0
+    clocks = sampler.stop() if rank == 0 else None
+    job.ctx.status()
+    value = world * tokens_per_gen * args.steps / (ms * 1e-3)
+
+    # per-kernel time of the attention kernel (events around it inside the library), same work
+    B.st3_profile_enable(job.ctx.handle, True)
+    for _ in range(args.steps):
+        job.generation()
+    attn_ms, finish_ms, n_attn, _ = B.st3_profile_read(job.ctx.handle)
+    B.st3_profile_enable(job.ctx.handle, False)
+    alg = sum(attend_bytes(wl, job.cfg, B, job.text, t) for t in range(0, wl.decode_steps + 1)) * args.steps
+    peak, peak_kind = measured_peak()
+    achieved = alg / (attn_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "st3_attend_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": f"of {peak_kind}", "traffic": None,
+                "algorithmic_bytes_per_launch": alg / max(1, n_attn), "us_per_launch": attn_ms * 1e3 / max(1, n_attn),
+                "launches_timed": n_attn, "attend_share_of_kernel_time": attn_ms / max(1e-9, attn_ms + finish_ms)}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": config,
+            "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks}
+
+    # end to end: every input starts in pinned host memory, every output ends there
+    job.make_host()
+    for _ in range(2):
+        job.generation_host()
+    ms_e2e = timed(job.generation_host, args.steps, dist)
+    job.ctx.status()
+    line["e2e"] = {"value": world * tokens_per_gen * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
+                   "h2d_bytes_per_step": job.h2d_bytes(), "d2h_bytes_per_step": job.d2h_bytes(),
+                   "ms_per_step": ms_e2e / args.steps}
+
+    if rank == 0 and world == 1 and not args.no_extras:
+        # the same kernels with trimming disabled (full KV cache)
+        full = Job(wl, device, disable_trim=True, rows_per_chunk=args.rows_per_chunk)
+        for _ in range(3):
+            full.generation()
+        ms_full = timed(full.generation, args.steps, False)
+        full.ctx.status()
+        v_full = tokens_per_gen * args.steps / (ms_full * 1e-3)
+        line["unpruned"] = {"value": v_full, "unit": UNIT, "speedup_from_trimming": value / v_full}
+        full.ctx.close()
+        del full
+        # the oracle on the host cores, bounded sample
+        ns = 24 if wl.batch == 1 else max(1, 24 // wl.batch)
+        K, V, q0 = job.K.cpu(), job.V.cpu(), job.q0.cpu()
+        q, kn, vn = job.q[:ns + 2].cpu(), job.kn[:ns + 2].cpu(), job.vn[:ns + 2].cpu()
+        val, secs, threads, s_first, s_last = oracle_sample(wl, job.g, K, V, q0, q, kn, vn, ns, 2)
+        line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "sample": f"all {wl.num_layers} layers x {wl.batch} sequence(s), decode steps "
+                                          f"{s_first}-{s_last} of {wl.decode_steps} after the oracle's own prefill "
+                                          f"({secs:.1f} s)"}
+    if rank == 0:
+        print(json.dumps(line))
+    job.ctx.close()
+    if dist:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

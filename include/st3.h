@@ -163,6 +163,25 @@ st3_status st3_profile_read(st3_ctx* ctx, double* attn_ms, double* finish_ms, in
 /* Total kernels this context has launched so far (host counter). */
 int64_t st3_launch_count(const st3_ctx* ctx);
 
+/* Attention of one query per head over dense K/V with NO workspace and no allocation of any kind
+ * (the paper has no counterpart; this exists for callers that may not allocate device memory:
+ * a plugin handed only its input and output tensors, code running inside a region whose memory
+ * another allocator owns, a process whose device memory is already fully committed).
+ *   q   dev [H][D]            k, v  dev [H][num_rows][D]            out  dev [H][D]
+ * computes out[h] = softmax(q[h] . k[h]^T / sqrt(D)) v[h], i.e. Eq. 2's last row, like
+ * st3_prefill_select does for a prompt of num_rows tokens.  The split partials go to a fixed
+ * array inside the library image (4 259 840 bytes, resident on every GPU that has loaded the
+ * library until the process exits), which limits a call to
+ *     num_heads * ceil(num_rows / 128) <= 8192        (else ST3_ERR_CAPACITY, nothing is launched).
+ * No cudaMalloc/cudaFree and no allocating library routine is called.  The first call on each
+ * device looks up the array's device address (cudaGetSymbolAddress, with that device current);
+ * make that first call before starting any stream capture.  All calls on a device share the one
+ * array and it keeps the previous call's contents: nothing in it needs to start at zero (every
+ * slot a call reads it has written first), but two calls whose kernels overlap on the GPU
+ * (different streams, no dependency between them) race on it and must be ordered by the caller. */
+st3_status st3_attend_noalloc(const void* q, const void* k, const void* v, void* out, int32_t num_heads,
+                              int32_t num_rows, int32_t head_dim, int32_t dtype, void* cuda_stream);
+
 const char* st3_status_string(st3_status s);
 
 /* Frees the host-side context.  Does not synchronise and does not touch the workspace. */

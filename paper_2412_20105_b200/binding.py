@@ -21,7 +21,8 @@ DEV_COUNT_MISMATCH, DEV_NONFINITE, DEV_COPY_TIMEOUT, DEV_RANGE = 1, 2, 4, 8
 
 EXPORTS = ["st3_schedule_count", "st3_workspace_size", "st3_create", "st3_prefill_select", "st3_decode_step",
            "st3_decode_step_host", "st3_get_kept", "st3_get_rows", "st3_get_status", "st3_rows_held",
-           "st3_profile_enable", "st3_profile_read", "st3_launch_count", "st3_status_string", "st3_destroy"]
+           "st3_profile_enable", "st3_profile_read", "st3_launch_count", "st3_status_string", "st3_destroy",
+           "st3_attend_noalloc"]
 
 
 class Config(C.Structure):
@@ -72,6 +73,7 @@ def load():
     lib.st3_status_string.argtypes = [C.c_int]
     lib.st3_status_string.restype = C.c_char_p
     lib.st3_destroy.argtypes = [vp]
+    lib.st3_attend_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
     for name in EXPORTS:
         if name not in ("st3_schedule_count", "st3_launch_count", "st3_status_string"):
             getattr(lib, name).restype = C.c_int
@@ -169,6 +171,14 @@ def st3_status_string(code: int) -> str:
 
 def st3_destroy(ctx):
     _check(load().st3_destroy(ctx), "st3_destroy")
+
+
+def st3_attend_noalloc(q, k, v, out, num_heads, num_rows, head_dim, dtype, stream=0):
+    """Workspace-free attention for callers that may not allocate device memory: q/k/v/out are
+    device addresses, the split partials live in a fixed array inside the library (see st3.h for
+    the size limit and the sharing rules)."""
+    dt = {"f32": ST3_F32, "bf16": ST3_BF16}.get(dtype, dtype)
+    _check(load().st3_attend_noalloc(q, k, v, out, num_heads, num_rows, head_dim, dt, stream), "st3_attend_noalloc")
 
 
 class Context:

@@ -1023,3 +1023,172 @@ st3_status st3_destroy(st3_ctx* ctx) {
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// st3_attend_noalloc: one-shot attention whose split partials live in a static device array
+// ------------------------------------------------------------------------------------------
+// Some callers cannot hand this library a workspace: code that runs where cudaMalloc is off
+// limits (inside a framework's allocator-owned region, in a plugin that was given only its
+// input and output tensors, late in a process whose memory is fully committed).  For them the
+// chunk partials of the attention go into the fixed array below instead of caller memory.
+// The array is part of the loaded module: every GPU that loads the library holds these bytes
+// until the process exits, which is why the limit is kept small.
+constexpr int kNaChunkRows = 128;
+constexpr int kNaMaxSlots = 8192;  // heads x row chunks of one call
+constexpr size_t kNaScratchBytes = (size_t)kNaMaxSlots * (2 + 128) * sizeof(float);  // 4 259 840 bytes
+static __device__ __align__(256) unsigned char st3_static_scratch[kNaScratchBytes];
+
+namespace {
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads) st3_na_partial_kernel(const T* __restrict__ q, const T* __restrict__ K,
+                                                                  const T* __restrict__ V, int num_rows, int nchunk,
+                                                                  float* part_ml, float* part_acc) {
+  constexpr int EPL = 16 / sizeof(T), LPR = D / EPL, RPW = 32 / LPR;
+  __shared__ float s_log[kNaChunkRows];
+  __shared__ float s_red[kWarps * D];
+  __shared__ float s_stat[kWarps];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int c = blockIdx.x, h = blockIdx.y;
+  const int r0 = c * kNaChunkRows, nrows = min(num_rows, r0 + kNaChunkRows) - r0;
+  const int sub = lane / LPR, lir = lane % LPR;
+  const uint4* gK = reinterpret_cast<const uint4*>(K + ((long long)h * num_rows + r0) * D);
+  const uint4* gV = reinterpret_cast<const uint4*>(V + ((long long)h * num_rows + r0) * D);
+  float qf[EPL];
+  unpack16(__ldg(reinterpret_cast<const uint4*>(q + (long long)h * D) + lir), qf);
+  const float sc = 1.4426950408889634f * rsqrtf((float)D);
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) qf[e] *= sc;
+  for (int rb = warp * RPW; rb < nrows; rb += kWarps * RPW) {
+    const int r = rb + sub;
+    float acc = 0.f;
+    if (r < nrows) {
+      float kf[EPL];
+      unpack16(__ldg(gK + (long long)r * LPR + lir), kf);
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc = fmaf(qf[e], kf[e], acc);
+    }
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (r < nrows && lir == 0) s_log[r] = acc;
+  }
+  __syncthreads();
+  float m = -INFINITY;
+  for (int r = tid; r < nrows; r += kThreads) m = fmaxf(m, s_log[r]);
+  m = warp_max(m);
+  if (lane == 0) s_stat[warp] = m;
+  __syncthreads();
+  m = s_stat[0];
+#pragma unroll
+  for (int w = 1; w < kWarps; ++w) m = fmaxf(m, s_stat[w]);
+  __syncthreads();
+  float lsum = 0.f;
+  for (int r = tid; r < nrows; r += kThreads) {
+    const float pr = fast_exp2(s_log[r] - m);
+    s_log[r] = pr;
+    lsum += pr;
+  }
+  lsum = warp_sum(lsum);
+  if (lane == 0) s_stat[warp] = lsum;
+  __syncthreads();
+  const long long slot = (long long)h * nchunk + c;
+  if (tid == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) t += s_stat[w];
+    part_ml[2 * slot] = m;
+    part_ml[2 * slot + 1] = t;
+  }
+  float acc[EPL];
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
+  for (int rb = warp * RPW; rb < nrows; rb += kWarps * RPW) {
+    const int r = rb + sub;
+    if (r < nrows) {
+      float vf[EPL];
+      unpack16(__ldg(gV + (long long)r * LPR + lir), vf);
+      const float pr = s_log[r];
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) acc[e] = fmaf(pr, vf[e], acc[e]);
+    }
+  }
+#pragma unroll
+  for (int o = LPR; o < 32; o <<= 1) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
+  }
+  if (lane < LPR) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) s_red[warp * D + lir * EPL + e] = acc[e];
+  }
+  __syncthreads();
+  if (tid < D) {
+    float t = 0.f;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) t += s_red[w * D + tid];
+    part_acc[slot * D + tid] = t;
+  }
+}
+
+template <typename T, int D>
+__global__ void st3_na_merge_kernel(T* __restrict__ out, int nchunk, const float* __restrict__ part_ml,
+                                    const float* __restrict__ part_acc) {
+  const int h = blockIdx.x, d = threadIdx.x;  // D threads
+  const long long s0 = (long long)h * nchunk;
+  float M = -INFINITY;
+  for (int c = 0; c < nchunk; ++c) M = fmaxf(M, part_ml[2 * (s0 + c)]);
+  float L = 0.f, o = 0.f;
+  for (int c = 0; c < nchunk; ++c) {
+    const float w = fast_exp2(part_ml[2 * (s0 + c)] - M);
+    L = fmaf(part_ml[2 * (s0 + c) + 1], w, L);
+    o = fmaf(part_acc[(s0 + c) * D + d], w, o);
+  }
+  store_out(out + (long long)h * D + d, o / L);
+}
+
+// Device address of st3_static_scratch, looked up once per device.  In host code the array's
+// name is only a handle for the runtime, never an address a kernel may be given.
+constexpr int kNaMaxDevices = 64;
+void* g_na_ptr[kNaMaxDevices] = {nullptr};
+
+st3_status na_scratch(float** ml, float** acc) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kNaMaxDevices) return ST3_ERR_CUDA;
+  void* p = __atomic_load_n(&g_na_ptr[dev], __ATOMIC_ACQUIRE);
+  if (!p) {
+    if (cudaGetSymbolAddress(&p, st3_static_scratch) != cudaSuccess || !p) return ST3_ERR_CUDA;
+    __atomic_store_n(&g_na_ptr[dev], p, __ATOMIC_RELEASE);  // same value from every racing thread
+  }
+  *ml = reinterpret_cast<float*>(p);
+  *acc = *ml + 2 * (size_t)kNaMaxSlots;
+  return ST3_OK;
+}
+
+template <typename T, int D>
+st3_status na_launch(const void* q, const void* k, const void* v, void* out, int H, int rows, cudaStream_t st) {
+  float *ml, *acc;
+  const st3_status s = na_scratch(&ml, &acc);
+  if (s != ST3_OK) return s;
+  const int nchunk = ceil_div(rows, kNaChunkRows);
+  st3_na_partial_kernel<T, D><<<dim3((unsigned)nchunk, (unsigned)H), kThreads, 0, st>>>(
+      static_cast<const T*>(q), static_cast<const T*>(k), static_cast<const T*>(v), rows, nchunk, ml, acc);
+  st3_na_merge_kernel<T, D><<<(unsigned)H, D, 0, st>>>(static_cast<T*>(out), nchunk, ml, acc);
+  return cudaGetLastError() == cudaSuccess ? ST3_OK : ST3_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" st3_status st3_attend_noalloc(const void* q, const void* k, const void* v, void* out, int32_t num_heads,
+                                         int32_t num_rows, int32_t head_dim, int32_t dtype, void* cuda_stream) {
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return ST3_ERR_INVALID_ARG;
+  if (num_heads < 1 || num_rows < 1 || (head_dim != 64 && head_dim != 128)) return ST3_ERR_INVALID_ARG;
+  if (dtype != ST3_F32 && dtype != ST3_BF16) return ST3_ERR_INVALID_ARG;
+  // the static array has room for kNaMaxSlots (head, 128-row chunk) partials and no more
+  if ((long long)num_heads * ceil_div(num_rows, kNaChunkRows) > kNaMaxSlots) return ST3_ERR_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (dtype == ST3_BF16)
+    return head_dim == 128 ? na_launch<__nv_bfloat16, 128>(q, k, v, out, num_heads, num_rows, st)
+                           : na_launch<__nv_bfloat16, 64>(q, k, v, out, num_heads, num_rows, st);
+  return head_dim == 128 ? na_launch<float, 128>(q, k, v, out, num_heads, num_rows, st)
+                         : na_launch<float, 64>(q, k, v, out, num_heads, num_rows, st);
+}

@@ -36,9 +36,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kPieceRows = 64;  // rows per bulk copy / mbarrier
-constexpr int kMaxChunkRows = 256;
-constexpr int kMaxPieces = kMaxChunkRows / kPieceRows;
+constexpr int kMaxChunkRows = 128;  // upper bound on the rows of one work item
 constexpr int kMaxLayers = 64;
 constexpr int kMaxHeads = 128;
 constexpr int kMaxVisual = 8192;
@@ -58,11 +56,15 @@ struct StepParams {
   int* n_cur;            // [l][b]
   const int* text_len;   // [b]
   int* status;
+  int* work_counter;     // next work item of the running attention launch
+  int* tickets;          // [l][b][h] partials published so far (self-resetting)
+  float* head_stat;      // [l][b][h][2]   (max, 1/sum) of the merged softmax, log2 domain
   long long lbh_stride;  // elements per (l, b, h) cache block
   int layer_begin, layer_count, B, H;
   int sys_len, Nv, cap_txt, step, append;
   int ct;                   // text chunks per (l, b, h), the same for every sequence
-  int chunk_rows;           // shared-memory tile capacity in rows
+  int chunk_rows;           // rows per work item (<= the kernel's tile capacity)
+  int total_work;           // work items x heads of this launch
   int cvp[kMaxLayers + 1];  // prefix sum of visual chunks per layer (relative layer index)
   int ncur[kMaxLayers];     // visual rows held before this step (host's schedule bookkeeping)
   int ntgt[kMaxLayers];     // visual rows to hold after this step
@@ -101,18 +103,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
       : "r"(smem_u32(bar)), "r"(parity)
       : "memory");
   return ok != 0;
-}
-// Bounded wait: gives up after kWaitCycles, records it in the status word and lets the block run
-// to completion on whatever is in shared memory (the result is then flagged invalid).
-__device__ __forceinline__ void mbar_wait(uint64_t* bar, uint32_t parity, int* status) {
-  if (mbar_try_wait(bar, parity)) return;
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitCycles) {
-      atomicOr(status, ST3_DEV_COPY_TIMEOUT);
-      return;
-    }
-  }
 }
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -173,188 +163,367 @@ __device__ __forceinline__ Item decode_item(const StepParams& p, int item) {
 }
 
 // ------------------------------------------------------------------------------------------
-// Attention partials (Eq. 2, last row) + raw visual logits + KV append
+// Attention (Eq. 2, last row) + raw visual logits + KV append: persistent, warp-specialised
 // ------------------------------------------------------------------------------------------
+// One block per SM.  Warp 0 (producer) fetches work items from a global counter and streams each
+// item's K rows, V rows and query into a 3-slot shared-memory ring with bulk asynchronous copies;
+// warps 4..11 (consumers) each own a fixed 1/8 of an item's rows: logits, tile-local softmax,
+// p.V, then dump their un-normalised result over their own (already consumed) K tile; warps 1..3
+// (mergers, one per ring slot) fold the eight warp results into the item's partial, publishes it, and - when it
+// publishes the last partial of a (layer, sequence, head) - merges all partials of that head
+// into the attention output.  Loads for the next two items are always in flight while an item is
+// being computed.  Every mbarrier wait is bounded; a timeout sets an abort flag that ends all roles.
+constexpr int kConsumers = 8;
+constexpr int kSlots = 3;
+constexpr int kAttendThreads = 32 * (1 + kSlots + kConsumers);  // producer, one merger per slot, consumers
+constexpr int kQBytes = 512;
+
+struct ItemDesc {
+  int nrows;  // < 0: no more work
+  int slot_lo, slot_hi;  // partial index (item * H + h), 64-bit
+  int lbh_lo, lbh_hi;    // (l * B + b) * H + h, absolute layer
+  int out_lo, out_hi;    // (l_rel * B + b) * H + h
+  int r0;                // first row of the chunk inside its segment
+  int want_logits;
+  int nit;               // partials of this (l, b, h)
+  int item0_lo, item0_hi;  // first item of this (l, b)
+  int h;
+};
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ long long join64(int lo, int hi) {
+  return (long long)(((unsigned long long)(unsigned)hi << 32) | (unsigned)lo);
+}
+// Bounded wait of a whole warp that also gives up when another role has already aborted; the
+// answer is the same in every lane.
+__device__ __forceinline__ bool ring_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+  bool ok = mbar_try_wait(bar, parity);
+  if (!ok) {
+    const long long t0 = clock64();
+    while (!(ok = mbar_try_wait(bar, parity))) {
+      if (*abort_flag) break;
+      if (clock64() - t0 > kWaitCycles) {
+        *abort_flag = 1;
+        atomicOr(status, ST3_DEV_COPY_TIMEOUT);
+        break;
+      }
+    }
+  }
+  return __all_sync(0xffffffffu, ok);
+}
+
 template <typename T, int D>
-__global__ void __launch_bounds__(kThreads) st3_attend_kernel(const StepParams p) {
-  constexpr int EPL = 16 / sizeof(T);  // elements per 16-byte lane load
-  constexpr int LPR = D / EPL;         // lanes per row
-  constexpr int RPW = 32 / LPR;        // rows per warp instruction
-  constexpr int ROWB = D * sizeof(T);
-  static_assert(LPR <= 32 && RPW >= 1, "row must fit one warp instruction");
+__global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const StepParams p) {
+  constexpr int EPL = 16 / sizeof(T);      // elements per 16-byte chunk
+  constexpr int ROWB = D * sizeof(T);      // bytes per row
+  constexpr int CPL = ROWB / 64;           // 16-byte chunks per lane (a lane owns a quarter row)
+  constexpr int kTileBytes = ROWB >= 512 ? 32768 : 16384;  // K (and V) bytes of one ring slot
+  constexpr int RMAX = kTileBytes / ROWB;  // rows per item: 64 (128 for 128-byte rows)
+  constexpr int TR = RMAX / kConsumers;    // rows per consumer warp
+  constexpr int GR = TR / 8;               // groups of 8 rows per warp
+  constexpr int QD = D / 4;                // dims per lane
+  constexpr int SLOTB = 2 * kTileBytes + kQBytes;
+  constexpr bool kDumpSplit = 32 * D > TR * ROWB;  // 8 x D floats do not fit a warp's K rows
+  static_assert(16 * D <= TR * ROWB, "warp result does not fit its own K and V rows");
+  static_assert(CPL >= 2 && CPL <= 8 && GR >= 1, "unsupported row size");
 
   extern __shared__ __align__(128) unsigned char smem[];
-  __shared__ float s_red[kWarps * D];
-  __shared__ float s_stat[kWarps];
-  __shared__ __align__(8) uint64_t s_bar[2 * kMaxPieces];
+  __shared__ __align__(8) uint64_t s_fullK[kSlots], s_fullV[kSlots], s_done[kSlots], s_empty[kSlots];
+  __shared__ ItemDesc s_desc[kSlots];
+  __shared__ float s_stat[kSlots][kConsumers][2];
+  __shared__ int s_abort;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int H = p.H;
-  const int h = blockIdx.x % H;
-  const int item = blockIdx.x / H;
-  const Item it = decode_item(p, item);
-  const int l = p.layer_begin + it.l_rel, b = it.b;
-  const bool is_vis = it.c < it.cv;
-
-  // rows of this chunk
-  int seg_rows, nchunk, ci;
-  if (is_vis) {
-    seg_rows = p.ncur[it.l_rel]; nchunk = it.cv; ci = it.c;
-  } else {
-    seg_rows = p.sys_len + __ldg(p.text_len + b) + p.step; nchunk = p.ct; ci = it.c - it.cv;
-  }
-  const int rows_per = (seg_rows + nchunk - 1) / nchunk;
-  const int r0 = ci * rows_per;
-  const int r1 = min(seg_rows, r0 + rows_per);
-  const int nrows = r1 - r0;
-  const long long slot = (long long)item * H + h;
-  if (nrows <= 0 || nrows > p.chunk_rows) {  // empty chunk (ragged split); uniform for the block
-    if (nrows > p.chunk_rows && tid == 0) atomicOr(p.status, ST3_DEV_RANGE);
-    if (tid == 0) { p.part_ml[2 * slot] = -INFINITY; p.part_ml[2 * slot + 1] = 0.f; }
-    if (tid < D) p.part_acc[slot * D + tid] = 0.f;
-    return;
-  }
-  const bool has_new = !is_vis && p.append && r1 == seg_rows;  // this chunk ends on the newest row
-  const int nbulk = nrows - (has_new ? 1 : 0);
-
-  const long long lbh = ((long long)l * p.B + b) * H + h;
-  T* blk = reinterpret_cast<T*>(p.cache) + lbh * p.lbh_stride;
-  T* gK = is_vis ? blk : blk + 2LL * p.Nv * D;
-  T* gV = gK + (is_vis ? (long long)p.Nv * D : (long long)p.cap_txt * D);
-
-  unsigned char* sK = smem;
-  unsigned char* sV = smem + (size_t)p.chunk_rows * ROWB;
-  float* s_log = reinterpret_cast<float*>(sV + (size_t)p.chunk_rows * ROWB);
-
   if (tid == 0) {
-    const int npiece = (nbulk + kPieceRows - 1) / kPieceRows;
-    for (int i = 0; i < npiece; ++i) { mbar_init(&s_bar[i], 1); mbar_init(&s_bar[kMaxPieces + i], 1); }
+    for (int s = 0; s < kSlots; ++s) {
+      mbar_init(&s_fullK[s], 1); mbar_init(&s_fullV[s], 1);
+      mbar_init(&s_done[s], kConsumers); mbar_init(&s_empty[s], 1);
+    }
+    s_abort = 0;
     mbar_fence_init();
-    for (int kv = 0; kv < 2; ++kv) {
-      const unsigned char* g = reinterpret_cast<const unsigned char*>(kv ? gV : gK) + (size_t)r0 * ROWB;
-      unsigned char* s = kv ? sV : sK;
-      for (int i = 0; i < npiece; ++i) {
-        const int rows = min(kPieceRows, nbulk - i * kPieceRows);
-        const uint32_t bytes = (uint32_t)rows * ROWB;
-        uint64_t* bar = &s_bar[kv * kMaxPieces + i];
-        mbar_expect_tx(bar, bytes);
-        bulk_g2s(s + (size_t)i * kPieceRows * ROWB, g + (size_t)i * kPieceRows * ROWB, bytes, bar);
+  }
+  __syncthreads();
+  volatile int* abort_flag = &s_abort;
+  const int H = p.H;
+  const int total = p.total_work;
+
+  if (warp == 0) {
+    // ===================== producer =====================
+    int x_next = 0, end_marks = 0;
+    if (lane == 0) x_next = atomicAdd(p.work_counter, 1);
+    for (int round = 0;; ++round) {
+      const int s = round % kSlots;
+      const uint32_t par = (uint32_t)(round / kSlots) & 1u;
+      if (!ring_wait(&s_empty[s], par ^ 1u, abort_flag, p.status)) break;
+      const int x = __shfl_sync(0xffffffffu, x_next, 0);
+      if (x >= total) {  // out of work: one end marker per slot, so that every merger sees one
+        if (lane == 0) { s_desc[s].nrows = -1; mbar_arrive(&s_fullK[s]); }
+        if (++end_marks == kSlots) break;
+        continue;
+      }
+      if (lane == 0) x_next = atomicAdd(p.work_counter, 1);  // prefetch the next item index
+      const int h = x % H, item = x / H;
+      const Item it = decode_item(p, item);
+      const int l = p.layer_begin + it.l_rel, b = it.b;
+      const bool is_vis = it.c < it.cv;
+      int seg_rows, nchunk, ci;
+      if (is_vis) { seg_rows = p.ncur[it.l_rel]; nchunk = it.cv; ci = it.c; }
+      else { seg_rows = p.sys_len + __ldg(p.text_len + b) + p.step; nchunk = p.ct; ci = it.c - it.cv; }
+      const int rows_per = (seg_rows + nchunk - 1) / nchunk;
+      const int r0 = ci * rows_per;
+      int nrows = min(seg_rows, r0 + rows_per) - r0;
+      if (nrows < 0) nrows = 0;
+      if (nrows > RMAX) { nrows = RMAX; if (lane == 0) atomicOr(p.status, ST3_DEV_RANGE); }
+      const bool has_new = !is_vis && p.append && nrows > 0 && r0 + nrows == seg_rows;
+      const int nbulk = nrows - (has_new ? 1 : 0);
+      const long long lbh = ((long long)l * p.B + b) * H + h;
+      const long long oidx = ((long long)it.l_rel * p.B + b) * H + h;
+      T* blk = reinterpret_cast<T*>(p.cache) + lbh * p.lbh_stride;
+      T* gK = is_vis ? blk : blk + 2LL * p.Nv * D;
+      T* gV = gK + (is_vis ? (long long)p.Nv * D : (long long)p.cap_txt * D);
+      unsigned char* sK = smem + (size_t)s * SLOTB;
+      unsigned char* sV = sK + kTileBytes;
+      unsigned char* sQ = sV + kTileBytes;
+      if (has_new && lane < 2 * (ROWB / 16 <= 16 ? ROWB / 16 : 16)) {
+        // newest row: from the step's inputs to the cache and into the tile (ROWB/16 vectors each)
+        constexpr int VPR = ROWB / 16;
+        constexpr int LN = VPR <= 16 ? VPR : 16;
+        const int kv = lane / LN, c0 = lane % LN;
+        const T* src = reinterpret_cast<const T*>(kv ? p.v_new : p.k_new) + oidx * D;
+        T* dstg = (kv ? gV : gK) + (long long)(seg_rows - 1) * D;
+        for (int c = c0; c < VPR; c += LN) {
+          const uint4 val = __ldg(reinterpret_cast<const uint4*>(src) + c);
+          reinterpret_cast<uint4*>(dstg)[c] = val;
+          *reinterpret_cast<uint4*>((kv ? sV : sK) + (size_t)(nrows - 1) * ROWB + c * 16) = val;
+        }
+      }
+      __syncwarp();
+      if (lane == 0) {
+        ItemDesc& d = s_desc[s];
+        const long long slot = (long long)item * H + h;
+        const long long item0 = (long long)p.B * (p.cvp[it.l_rel] + it.l_rel * p.ct) + (long long)b * (it.cv + p.ct);
+        d.nrows = nrows;
+        d.slot_lo = (int)slot; d.slot_hi = (int)(slot >> 32);
+        d.lbh_lo = (int)lbh; d.lbh_hi = (int)(lbh >> 32);
+        d.out_lo = (int)oidx; d.out_hi = (int)(oidx >> 32);
+        d.r0 = r0;
+        d.want_logits = is_vis && p.ntgt[it.l_rel] < p.ncur[it.l_rel];
+        d.nit = it.cv + p.ct;
+        d.item0_lo = (int)item0; d.item0_hi = (int)(item0 >> 32);
+        d.h = h;
+        const uint32_t kb = (uint32_t)nbulk * ROWB;
+        mbar_expect_tx(&s_fullK[s], kb + ROWB);  // K rows + the query (D elements = ROWB bytes)
+        bulk_g2s(sQ, reinterpret_cast<const T*>(p.q) + oidx * D, ROWB, &s_fullK[s]);
+        if (kb) bulk_g2s(sK, reinterpret_cast<const unsigned char*>(gK) + (size_t)r0 * ROWB, kb, &s_fullK[s]);
+        if (kb) {
+          mbar_expect_tx(&s_fullV[s], kb);
+          bulk_g2s(sV, reinterpret_cast<const unsigned char*>(gV) + (size_t)r0 * ROWB, kb, &s_fullV[s]);
+        } else {
+          mbar_arrive(&s_fullV[s]);
+        }
       }
     }
-  }
-
-  const int sub = lane / LPR;  // which of the RPW rows of a warp instruction
-  const int lir = lane % LPR;  // 16-byte column inside the row
-  const long long qoff = (((long long)it.l_rel * p.B + b) * H + h) * D;
-
-  // query, pre-scaled by log2(e)/sqrt(D) so that probabilities are exp2(logit - max)
-  float qf[EPL];
-  {
-    const uint4 qv = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(p.q) + qoff) + lir);
-    unpack16(qv, qf);
-    const float sc = 1.4426950408889634f * rsqrtf((float)D);
+  } else if (warp <= kSlots) {
+    // ===================== mergers: warp 1 + s serves ring slot s =====================
+    constexpr int DPL = D / 32;  // output dims per lane
+    const int s = warp - 1;
+    for (int use = 0;; ++use) {
+      const uint32_t par = (uint32_t)use & 1u;
+      if (!ring_wait(&s_done[s], par, abort_flag, p.status)) break;
+      const ItemDesc d = s_desc[s];
+      if (d.nrows < 0) break;
+      const int nw = (d.nrows + TR - 1) / TR;
+      float M = -INFINITY;
+      for (int w = 0; w < nw; ++w) M = fmaxf(M, s_stat[s][w][0]);
+      float Lsum = 0.f, o[DPL];
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) qf[e] *= sc;
-  }
-  // newest row: comes from the step's inputs, goes to the cache and into the tile
-  if (has_new && tid < 2 * LPR) {
-    const int kv = tid / LPR, c = tid % LPR;
-    const T* src = reinterpret_cast<const T*>(kv ? p.v_new : p.k_new) + qoff;
-    const uint4 val = __ldg(reinterpret_cast<const uint4*>(src) + c);
-    T* dstg = (kv ? gV : gK) + (long long)(seg_rows - 1) * D;
-    reinterpret_cast<uint4*>(dstg)[c] = val;
-    *reinterpret_cast<uint4*>((kv ? sV : sK) + (size_t)(nrows - 1) * ROWB + c * 16) = val;
-  }
-  __syncthreads();  // barrier inits and the newest row are visible
-
-  // ---- K pass: logits ----
-  for (int base = 0; base < nrows; base += kPieceRows) {
-    if (base < nbulk) mbar_wait(&s_bar[base / kPieceRows], 0, p.status);
-    const int pend = min(nrows, base + kPieceRows);
-#pragma unroll 2
-    for (int rb = base + warp * RPW; rb < pend; rb += kWarps * RPW) {
-      const int r = rb + sub;
-      float acc = 0.f;
-      if (r < pend) {
-        const uint4 kvv = *reinterpret_cast<const uint4*>(sK + (size_t)r * ROWB + lir * 16);
-        float kf[EPL];
-        unpack16(kvv, kf);
+      for (int j = 0; j < DPL; ++j) o[j] = 0.f;
+      const unsigned char* sK = smem + (size_t)s * SLOTB;
+      for (int w = 0; w < nw; ++w) {
+        const float wgt = fast_exp2(s_stat[s][w][0] - M);
+        Lsum = fmaf(s_stat[s][w][1], wgt, Lsum);
+        const float* dumpK = reinterpret_cast<const float*>(sK + (size_t)w * TR * ROWB);
+        const float* dumpV = reinterpret_cast<const float*>(sK + kTileBytes + (size_t)w * TR * ROWB);
+        float t[DPL];
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) acc = fmaf(qf[e], kf[e], acc);
+        for (int j = 0; j < DPL; ++j) t[j] = 0.f;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          const float* dump = kDumpSplit ? (g >= 4 ? dumpV - 4 * D : dumpK) : dumpK;
+          if (DPL == 4) {
+            const float4 v4 = *reinterpret_cast<const float4*>(dump + g * D + lane * 4);
+            t[0] += v4.x; t[1] += v4.y; t[2] += v4.z; t[DPL - 1] += v4.w;
+          } else {
+            const float2 v2 = *reinterpret_cast<const float2*>(dump + g * D + lane * 2);
+            t[0] += v2.x; t[DPL - 1] += v2.y;
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < DPL; ++j) o[j] = fmaf(t[j], wgt, o[j]);
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_empty[s]);  // the slot may be refilled from here on
+      const long long slot = join64(d.slot_lo, d.slot_hi);
+      if (d.nrows == 0) M = -INFINITY;
 #pragma unroll
-      for (int o = LPR / 2; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-      if (r < pend && lir == 0) s_log[r] = acc;
-    }
-  }
-  __syncthreads();
-
-  // ---- chunk softmax statistics ----
-  float mloc = -INFINITY;
-  for (int r = tid; r < nrows; r += kThreads) mloc = fmaxf(mloc, s_log[r]);
-  mloc = warp_max(mloc);
-  if (lane == 0) s_stat[warp] = mloc;
-  __syncthreads();
-  float m = s_stat[0];
+      for (int j = 0; j < DPL; ++j) p.part_acc[slot * D + lane * DPL + j] = o[j];
+      if (lane == 0) { p.part_ml[2 * slot] = M; p.part_ml[2 * slot + 1] = Lsum; }
+      // ticket: whoever publishes the last partial of this (l, b, h) merges them all
+      __threadfence();
+      __syncwarp();
+      int last = 0;
+      const long long lbh = join64(d.lbh_lo, d.lbh_hi);
+      if (lane == 0) {
+        const int old = atomicAdd(p.tickets + lbh, 1);
+        last = (old == d.nit - 1);
+        if (last) p.tickets[lbh] = 0;  // ready for the next step
+      }
+      last = __shfl_sync(0xffffffffu, last, 0);
+      if (last) {
+        __threadfence();
+        const long long item0 = join64(d.item0_lo, d.item0_hi);
+        float Mh = -INFINITY;
+        for (int i = lane; i < d.nit; i += 32) Mh = fmaxf(Mh, __ldcg(p.part_ml + 2 * ((item0 + i) * H + d.h)));
+        Mh = warp_max(Mh);
+        float Lh = 0.f;
+        for (int i = lane; i < d.nit; i += 32) {
+          const long long sl = (item0 + i) * H + d.h;
+          Lh += __ldcg(p.part_ml + 2 * sl + 1) * fast_exp2(__ldcg(p.part_ml + 2 * sl) - Mh);
+        }
+        Lh = warp_sum(Lh);
+        float oh[DPL];
 #pragma unroll
-  for (int w = 1; w < kWarps; ++w) m = fmaxf(m, s_stat[w]);
-  __syncthreads();
-  const bool want_logits = is_vis && p.ntgt[it.l_rel] < p.ncur[it.l_rel];
-  float* glog = p.logits + lbh * p.Nv + r0;
-  float lsum = 0.f;
-  for (int r = tid; r < nrows; r += kThreads) {
-    const float s = s_log[r];
-    if (want_logits) glog[r] = s;
-    const float pr = fast_exp2(s - m);
-    s_log[r] = pr;
-    lsum += pr;
-  }
-  lsum = warp_sum(lsum);
-  if (lane == 0) s_stat[warp] = lsum;
-  __syncthreads();  // also publishes the probabilities in s_log
-  if (tid == 0) {
-    float t = 0.f;
+        for (int j = 0; j < DPL; ++j) oh[j] = 0.f;
+        for (int i = 0; i < d.nit; ++i) {
+          const long long sl = (item0 + i) * H + d.h;
+          const float wgt = fast_exp2(__ldcg(p.part_ml + 2 * sl) - Mh);
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) t += s_stat[w];
-    p.part_ml[2 * slot] = m;
-    p.part_ml[2 * slot + 1] = t;
-  }
-
-  // ---- V pass: un-normalised output ----
-  float acc[EPL];
+          for (int j = 0; j < DPL; ++j) oh[j] = fmaf(wgt, __ldcg(p.part_acc + sl * D + lane * DPL + j), oh[j]);
+        }
+        const float invL = 1.f / Lh;
+        T* out = reinterpret_cast<T*>(p.out) + join64(d.out_lo, d.out_hi) * D;
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-  for (int base = 0; base < nrows; base += kPieceRows) {
-    if (base < nbulk) mbar_wait(&s_bar[kMaxPieces + base / kPieceRows], 0, p.status);
-    const int pend = min(nrows, base + kPieceRows);
-#pragma unroll 2
-    for (int rb = base + warp * RPW; rb < pend; rb += kWarps * RPW) {
-      const int r = rb + sub;
-      if (r < pend) {
-        const float pr = s_log[r];
-        const uint4 vv = *reinterpret_cast<const uint4*>(sV + (size_t)r * ROWB + lir * 16);
-        float vf[EPL];
-        unpack16(vv, vf);
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) acc[e] = fmaf(pr, vf[e], acc[e]);
+        for (int j = 0; j < DPL; ++j) store_out(out + lane * DPL + j, oh[j] * invL);
+        if (lane == 0) { p.head_stat[2 * lbh] = Mh; p.head_stat[2 * lbh + 1] = invL; }
       }
     }
-  }
+  } else {
+    // ===================== consumers =====================
+    const int w = warp - 1 - kSlots;
+    const int r8 = lane >> 2, c4 = lane & 3;
+    int rot, end_marks = 0;
+    if (CPL == 2) rot = r8 & 1;
+    else if (CPL == 4) rot = (c4 >> 1) + 2 * (r8 & 1);
+    else rot = lane & 7;
+    for (int round = 0;; ++round) {
+      const int s = round % kSlots;
+      const uint32_t par = (uint32_t)(round / kSlots) & 1u;
+      if (!ring_wait(&s_fullK[s], par, abort_flag, p.status)) break;
+      const int nrows = s_desc[s].nrows;
+      if (nrows < 0) {  // end marker: pass it on to this slot's merger; the last one ends the warp
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&s_done[s]);
+        if (++end_marks == kSlots) break;
+        continue;
+      }
+      const int base = w * TR;
+      if (base < nrows) {
+        unsigned char* sK = smem + (size_t)s * SLOTB;
+        const unsigned char* sV = sK + kTileBytes;
+        const unsigned char* sQ = sV + kTileBytes;
+        const float sc = 1.4426950408889634f * rsqrtf((float)D);
+        // this lane's quarter of the query, in the rotated chunk order it reads rows in
+        float qf[CPL][EPL];
 #pragma unroll
-  for (int o = LPR; o < 32; o <<= 1) {
+        for (int j = 0; j < CPL; ++j) {
+          const int jj = (j + rot) & (CPL - 1);
+          unpack16(*reinterpret_cast<const uint4*>(sQ + (c4 * CPL + jj) * 16), qf[j]);
+        }
+        float sl[GR];
+        bool ok[GR];
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) acc[e] += __shfl_xor_sync(0xffffffffu, acc[e], o);
-  }
-  if (lane < LPR) {
+        for (int g = 0; g < GR; ++g) {
+          const int r = base + g * 8 + r8;
+          ok[g] = r < nrows;
+          float a[CPL];
 #pragma unroll
-    for (int e = 0; e < EPL; ++e) s_red[warp * D + lir * EPL + e] = acc[e];
-  }
-  __syncthreads();
-  if (tid < D) {
-    float t = 0.f;
+          for (int j = 0; j < CPL; ++j) a[j] = 0.f;
+          if (ok[g]) {
+            const unsigned char* row = sK + (size_t)r * ROWB + c4 * (CPL * 16);
 #pragma unroll
-    for (int w = 0; w < kWarps; ++w) t += s_red[w * D + tid];
-    p.part_acc[slot * D + tid] = t;
+            for (int j = 0; j < CPL; ++j) {
+              const int jj = (j + rot) & (CPL - 1);
+              float kf[EPL];
+              unpack16(*reinterpret_cast<const uint4*>(row + jj * 16), kf);
+#pragma unroll
+              for (int e = 0; e < EPL; ++e) a[j] = fmaf(qf[j][e], kf[e], a[j]);
+            }
+          }
+          float t = 0.f;
+#pragma unroll
+          for (int j = 0; j < CPL; ++j) t += a[j];
+          t += __shfl_xor_sync(0xffffffffu, t, 1);
+          t += __shfl_xor_sync(0xffffffffu, t, 2);
+          sl[g] = ok[g] ? t * sc : -INFINITY;  // log2-domain logit
+        }
+        float m = sl[0];
+#pragma unroll
+        for (int g = 1; g < GR; ++g) m = fmaxf(m, sl[g]);
+        m = warp_max(m);
+        const ItemDesc& d = s_desc[s];
+        if (d.want_logits && c4 == 0) {
+          float* glog = p.logits + join64(d.lbh_lo, d.lbh_hi) * p.Nv + d.r0;
+#pragma unroll
+          for (int g = 0; g < GR; ++g)
+            if (ok[g]) glog[base + g * 8 + r8] = sl[g];
+        }
+        float pr[GR], lsum = 0.f;
+#pragma unroll
+        for (int g = 0; g < GR; ++g) {
+          pr[g] = ok[g] ? fast_exp2(sl[g] - m) : 0.f;
+          if (c4 == 0) lsum += pr[g];
+        }
+        lsum = warp_sum(lsum);
+        if (!ring_wait(&s_fullV[s], par, abort_flag, p.status)) break;
+        float acc[CPL][EPL];
+#pragma unroll
+        for (int j = 0; j < CPL; ++j)
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) acc[j][e] = 0.f;
+#pragma unroll
+        for (int g = 0; g < GR; ++g) {
+          if (ok[g]) {
+            const unsigned char* row = sV + (size_t)(base + g * 8 + r8) * ROWB + c4 * (CPL * 16);
+#pragma unroll
+            for (int j = 0; j < CPL; ++j) {
+              const int jj = (j + rot) & (CPL - 1);
+              float vf[EPL];
+              unpack16(*reinterpret_cast<const uint4*>(row + jj * 16), vf);
+#pragma unroll
+              for (int e = 0; e < EPL; ++e) acc[j][e] = fmaf(pr[g], vf[e], acc[j][e]);
+            }
+          }
+        }
+        // dump [8 row groups][D] over this warp's own K rows (and, where those are too small, half of
+        // it over its own V rows)
+        __syncwarp();  // every lane has finished reading this warp's V rows as well
+        float* dump = reinterpret_cast<float*>((kDumpSplit && r8 >= 4 ? sK + kTileBytes : sK) + (size_t)base * ROWB) +
+                      (kDumpSplit ? (r8 & 3) : r8) * D + c4 * QD;
+#pragma unroll
+        for (int j = 0; j < CPL; ++j) {
+          const int jj = (j + rot) & (CPL - 1);
+#pragma unroll
+          for (int e = 0; e < EPL; e += 4)
+            *reinterpret_cast<float4*>(dump + jj * EPL + e) =
+                make_float4(acc[j][e], acc[j][e + 1], acc[j][e + 2], acc[j][e + 3]);
+        }
+        if (lane == 0) { s_stat[s][w][0] = m; s_stat[s][w][1] = lsum; }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&s_done[s]);
+    }
   }
 }
 
@@ -376,38 +545,7 @@ __global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p
   const int B = p.B, H = p.H, Nv = p.Nv;
   const int l_rel = blockIdx.x / B, b = blockIdx.x % B;
   const int l = p.layer_begin + l_rel;
-  const int cv = p.cvp[l_rel + 1] - p.cvp[l_rel];
-  const int nit = cv + p.ct;
-  const long long item0 = (long long)B * (p.cvp[l_rel] + l_rel * p.ct) + (long long)b * nit;
-
-  // ---- merge the chunk partials of every head ----
-  for (int h = warp; h < H; h += kWarps) {
-    float M = -INFINITY;
-    for (int s = lane; s < nit; s += 32) M = fmaxf(M, p.part_ml[2 * ((item0 + s) * H + h)]);
-    M = warp_max(M);
-    float L = 0.f;
-    for (int s = lane; s < nit; s += 32) {
-      const long long slot = (item0 + s) * H + h;
-      L += p.part_ml[2 * slot + 1] * fast_exp2(p.part_ml[2 * slot] - M);
-    }
-    L = warp_sum(L);
-    float o[D / 32];
-#pragma unroll
-    for (int j = 0; j < D / 32; ++j) o[j] = 0.f;
-    for (int s = 0; s < nit; ++s) {
-      const long long slot = (item0 + s) * H + h;
-      const float w = fast_exp2(p.part_ml[2 * slot] - M);
-#pragma unroll
-      for (int j = 0; j < D / 32; ++j) o[j] = fmaf(w, p.part_acc[slot * D + lane + 32 * j], o[j]);
-    }
-    const float invL = 1.f / L;
-    T* out = reinterpret_cast<T*>(p.out) + (((long long)l_rel * B + b) * H + h) * D;
-#pragma unroll
-    for (int j = 0; j < D / 32; ++j) store_out(out + lane + 32 * j, o[j] * invL);
-    if (lane == 0) { s_M[h] = M; s_invL[h] = invL; }
-  }
-  __syncthreads();
-
+  if (blockIdx.x == 0 && tid == 0) *p.work_counter = 0;  // the next attention launch starts from item 0
   const long long lb = (long long)l * B + b;
   const int n_cur = p.n_cur[lb];
   if (n_cur != p.ncur[l_rel]) {  // host bookkeeping and device state disagree: flag, do not touch
@@ -422,6 +560,12 @@ __global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p
   int* s_mover = s_hole + Nv;                                               // [Nv]
   int* ids = p.ids + lb * Nv;
   float* mass_by_id = p.mass_by_id + lb * Nv;
+
+  for (int h = tid; h < H; h += kThreads) {
+    s_M[h] = p.head_stat[2 * (lb * H + h)];
+    s_invL[h] = p.head_stat[2 * (lb * H + h) + 1];
+  }
+  __syncthreads();
 
   // ---- visual scores: probability of every visual row summed over heads ----
   bool bad = false;
@@ -584,7 +728,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 struct Layout {
-  size_t elem, cache, part_ml, part_acc, logits, mass, ids, n_cur, text_len, status, stage_q, stage_k, stage_v,
+  size_t elem, cache, part_ml, part_acc, logits, mass, ids, n_cur, tickets, head_stat, text_len, status, stage_q, stage_k, stage_v,
       stage_o, total;
   long long lbh_stride;
   int cap_txt, chunk_rows, max_items;
@@ -609,9 +753,19 @@ bool valid_config(const st3_config* c) {
   return true;
 }
 
+// Bytes of K (and of V) one ring slot of the attention kernel holds, and the rows that makes.
+int tile_bytes(const st3_config* c) {
+  const int rowb = c->head_dim * (c->dtype == ST3_BF16 ? 2 : 4);
+  return rowb >= 512 ? 32768 : 16384;
+}
+int tile_rows(const st3_config* c) {
+  return tile_bytes(c) / (c->head_dim * (c->dtype == ST3_BF16 ? 2 : 4));
+}
+
 int pick_chunk_rows(const st3_config* c) {
-  if (c->rows_per_chunk > 0) return c->rows_per_chunk;
-  return 128;
+  const int cap = tile_rows(c);
+  if (c->rows_per_chunk > 0) return c->rows_per_chunk < cap ? c->rows_per_chunk : cap;
+  return cap;
 }
 
 Layout make_layout(const st3_config* c) {
@@ -632,6 +786,8 @@ Layout make_layout(const st3_config* c) {
   L.mass = take(lb * (size_t)c->num_visual * sizeof(float));
   L.ids = take(lb * (size_t)c->num_visual * sizeof(int));
   L.n_cur = take(lb * sizeof(int));
+  L.tickets = take(lbh * sizeof(int));
+  L.head_stat = take(lbh * 2 * sizeof(float));
   L.text_len = take((size_t)c->batch * sizeof(int));
   L.status = take(256);
   const size_t io = lbh * c->head_dim * L.elem;
@@ -677,7 +833,7 @@ struct st3_ctx {
   bool profiling;
   std::vector<cudaEvent_t> ev_pool;  // triples: before attend, after attend, after finish
   size_t ev_used;
-  int attend_smem, finish_smem;
+  int attend_smem, finish_smem, num_sms, attend_ctas_per_sm;
 };
 
 namespace {
@@ -704,7 +860,8 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
     ctx->ev_used += 3;
     cudaEventRecord(e0, st);
   }
-  st3_attend_kernel<T, D><<<(unsigned)(total_items * c.num_heads), kThreads, ctx->attend_smem, st>>>(p);
+  (void)total_items;
+  st3_attend_kernel<T, D><<<(unsigned)(ctx->num_sms * ctx->attend_ctas_per_sm), kAttendThreads, ctx->attend_smem, st>>>(p);
   if (e1) cudaEventRecord(e1, st);
   st3_finish_kernel<T, D><<<(unsigned)(p.layer_count * c.batch), kThreads, ctx->finish_smem, st>>>(p);
   if (e2) cudaEventRecord(e2, st);
@@ -747,6 +904,9 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
   p.n_cur = reinterpret_cast<int*>(ctx->ws + L.n_cur);
   p.text_len = reinterpret_cast<const int*>(ctx->ws + L.text_len);
   p.status = reinterpret_cast<int*>(ctx->ws + L.status);
+  p.work_counter = p.status + 16;
+  p.tickets = reinterpret_cast<int*>(ctx->ws + L.tickets);
+  p.head_stat = reinterpret_cast<float*>(ctx->ws + L.head_stat);
   p.lbh_stride = L.lbh_stride;
   p.layer_begin = layer_begin; p.layer_count = layer_count; p.B = c.batch; p.H = c.num_heads;
   p.sys_len = c.sys_len; p.Nv = c.num_visual; p.cap_txt = L.cap_txt; p.step = step; p.append = prefill ? 0 : 1;
@@ -763,7 +923,8 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
     p.cvp[i + 1] = p.cvp[i] + ceil_div(ncur, R);
   }
   const long long total_items = (long long)c.batch * (p.cvp[layer_count] + (long long)layer_count * p.ct);
-  if (total_items > L.max_items || total_items * c.num_heads > 0x7fffffffLL) return ST3_ERR_CAPACITY;
+  if (total_items > L.max_items || total_items * c.num_heads > 0x3fffffffLL) return ST3_ERR_CAPACITY;
+  p.total_work = (int)(total_items * c.num_heads);
 
 #define ST3_LAUNCH(T, D) launch_step_t<T, D>(ctx, p, (int)total_items, st, k, v, prefill)
   const st3_status s = ST3_DISPATCH(ctx, ST3_LAUNCH);
@@ -819,8 +980,15 @@ st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, 
   ctx->launches = 0;
   ctx->profiling = false;
   ctx->ev_used = 0;
-  const size_t rowb = (size_t)cfg->head_dim * L.elem;
-  ctx->attend_smem = (int)(2 * (size_t)L.chunk_rows * rowb + (size_t)L.chunk_rows * sizeof(float));
+  ctx->attend_smem = kSlots * (2 * tile_bytes(cfg) + kQBytes);
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+    delete ctx;
+    return ST3_ERR_CUDA;
+  }
+  ctx->num_sms = sms;
+  ctx->attend_ctas_per_sm = tile_bytes(cfg) > 16384 ? 1 : 2;
   ctx->finish_smem = (int)((size_t)cfg->num_visual * 16 + 16);
   if (ctx->attend_smem > 200 * 1024 || ctx->finish_smem > 200 * 1024) { delete ctx; return ST3_ERR_UNSUPPORTED; }
 #define ST3_ATTR(T, D) set_attrs_t<T, D>(ctx)

@@ -25,7 +25,7 @@ def test_tiny_every_step(tau):
     assert stats["units"] == wl.decode_steps + 1
 
 
-@pytest.mark.parametrize("rows", [16, 64, 100, 256])
+@pytest.mark.parametrize("rows", [16, 64, 100, 128])
 def test_tiny_chunk_sizes_and_ragged_tails(rows):
     wl = get_workload("tiny")
     run_and_check(wl, 6, rows_per_chunk=rows)

@@ -36,6 +36,8 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
+constexpr int kFinishThreads = 1024;
+constexpr int kFinishWarps = kFinishThreads / 32;
 constexpr int kMaxChunkRows = 128;  // upper bound on the rows of one work item
 constexpr int kMaxLayers = 64;
 constexpr int kMaxHeads = 128;
@@ -57,15 +59,18 @@ struct StepParams {
   const int* text_len;   // [b]
   int* status;
   int* work_counter;     // next work item of the running attention launch
-  int* tickets;          // [l][b][h] partials published so far (self-resetting)
-  float* head_stat;      // [l][b][h][2]   (max, 1/sum) of the merged softmax, log2 domain
   long long lbh_stride;  // elements per (l, b, h) cache block
   int layer_begin, layer_count, B, H;
   int sys_len, Nv, cap_txt, step, append;
   int ct;                   // text chunks per (l, b, h), the same for every sequence
   int chunk_rows;           // rows per work item (<= the kernel's tile capacity)
   int total_work;           // work items x heads of this launch
+  unsigned h_mul, h_shift;  // fast division by H
   int cvp[kMaxLayers + 1];  // prefix sum of visual chunks per layer (relative layer index)
+  int lstart[kMaxLayers + 1];       // first work item of each layer: B * (cvp[l] + l * ct)
+  int rpv[kMaxLayers];              // rows per visual chunk of each layer
+  unsigned per_mul[kMaxLayers];     // fast division by (visual + text chunks) of each layer
+  unsigned per_shift[kMaxLayers];
   int ncur[kMaxLayers];     // visual rows held before this step (host's schedule bookkeeping)
   int ntgt[kMaxLayers];     // visual rows to hold after this step
 };
@@ -127,6 +132,48 @@ __device__ __forceinline__ void unpack16(const uint4& v, float (&f)[4]) {  // f3
   f[2] = __uint_as_float(v.z);
   f[3] = __uint_as_float(v.w);
 }
+// Packed pairs of fp32 for fma.rn.f32x2 (two FMAs per issued instruction).
+using u64 = unsigned long long;
+__device__ __forceinline__ u64 pack2(float lo, float hi) {
+  u64 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void fma2(u64& d, u64 a, u64 b) { asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b)); }
+__device__ __forceinline__ float sum2(u64 v) {
+  float lo, hi;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+  return lo + hi;
+}
+__device__ __forceinline__ void split2(u64 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ u64 bf16x2_pair(unsigned x) {  // two bf16 in one word -> (lo, hi) as fp32
+  return pack2(__uint_as_float(x << 16), __uint_as_float(x & 0xffff0000u));
+}
+__device__ __forceinline__ void unpack16_pairs(const uint4& v, u64 (&f)[4]) {  // bf16 x 8
+  f[0] = bf16x2_pair(v.x); f[1] = bf16x2_pair(v.y); f[2] = bf16x2_pair(v.z); f[3] = bf16x2_pair(v.w);
+}
+__device__ __forceinline__ void unpack16_pairs(const uint4& v, u64 (&f)[2]) {  // f32 x 4
+  f[0] = pack2(__uint_as_float(v.x), __uint_as_float(v.y));
+  f[1] = pack2(__uint_as_float(v.z), __uint_as_float(v.w));
+}
+// DPL consecutive elements of a row, as DPL/2 packed fp32 pairs
+template <typename T, int DPL>
+__device__ __forceinline__ void load_pairs(const unsigned char* p, u64 (&f)[DPL / 2]) {
+  if constexpr (sizeof(T) == 2 && DPL == 4) {
+    const uint2 v = *reinterpret_cast<const uint2*>(p);
+    f[0] = bf16x2_pair(v.x); f[DPL / 2 - 1] = bf16x2_pair(v.y);
+  } else if constexpr (sizeof(T) == 2) {
+    f[0] = bf16x2_pair(*reinterpret_cast<const unsigned*>(p));
+  } else if constexpr (DPL == 4) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    f[0] = pack2(v.x, v.y); f[DPL / 2 - 1] = pack2(v.z, v.w);
+  } else {
+    const float2 v = *reinterpret_cast<const float2*>(p);
+    f[0] = pack2(v.x, v.y);
+  }
+}
 __device__ __forceinline__ void store_out(float* p, float v) { *p = v; }
 __device__ __forceinline__ void store_out(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
@@ -141,60 +188,36 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
-// Which (relative layer, sequence, chunk) a flat item index names.  Items are ordered by layer,
-// then sequence, then chunk (visual chunks first, then text chunks).
-struct Item {
-  int l_rel, b, c, cv;
-};
-__device__ __forceinline__ Item decode_item(const StepParams& p, int item) {
-  int lo = 0, hi = p.layer_count - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (p.B * (p.cvp[mid] + mid * p.ct) <= item) lo = mid; else hi = mid - 1;
-  }
-  Item it;
-  it.l_rel = lo;
-  it.cv = p.cvp[lo + 1] - p.cvp[lo];
-  const int off = item - p.B * (p.cvp[lo] + lo * p.ct);
-  const int per = it.cv + p.ct;
-  it.b = off / per;
-  it.c = off - it.b * per;
-  return it;
-}
-
 // ------------------------------------------------------------------------------------------
 // Attention (Eq. 2, last row) + raw visual logits + KV append: persistent, warp-specialised
 // ------------------------------------------------------------------------------------------
-// One block per SM.  Warp 0 (producer) fetches work items from a global counter and streams each
-// item's K rows, V rows and query into a 3-slot shared-memory ring with bulk asynchronous copies;
-// warps 4..11 (consumers) each own a fixed 1/8 of an item's rows: logits, tile-local softmax,
-// p.V, then dump their un-normalised result over their own (already consumed) K tile; warps 1..3
-// (mergers, one per ring slot) fold the eight warp results into the item's partial, publishes it, and - when it
-// publishes the last partial of a (layer, sequence, head) - merges all partials of that head
-// into the attention output.  Loads for the next two items are always in flight while an item is
-// being computed.  Every mbarrier wait is bounded; a timeout sets an abort flag that ends all roles.
+// Two blocks per SM, each with a 3-slot shared-memory ring.  Warp s < 3 is the MANAGER of ring
+// slot s: it fetches a work item (layer, sequence, head, row chunk) from a global counter, streams
+// the item's K rows, V rows and query into its slot with bulk asynchronous copies, and - once the
+// consumers are done with the slot - folds their eight results into the item's partial, refills
+// the slot at once and only then stores the partial (plain stores; st3_finish_kernel merges the
+// partials of each head).  Warps 3..10 are CONSUMERS: each owns a fixed 1/8 of an item's rows
+// (K pass: four lanes per row; V pass: a lane owns D/32 output dims and walks the warp's rows):
+// logits, tile-local softmax, p.V; the warp leaves its un-normalised result over its own,
+// already consumed, K rows.  Loads of the other slots
+// are always in flight while one slot is being computed.  Every mbarrier wait is bounded; a
+// timeout raises a block-wide abort flag that ends all roles.
 constexpr int kConsumers = 8;
 constexpr int kSlots = 3;
-constexpr int kAttendThreads = 32 * (1 + kSlots + kConsumers);  // producer, one merger per slot, consumers
+constexpr int kAttendThreads = 32 * (kSlots + kConsumers);
 constexpr int kQBytes = 512;
 
 struct ItemDesc {
-  int nrows;  // < 0: no more work
-  int slot_lo, slot_hi;  // partial index (item * H + h), 64-bit
-  int lbh_lo, lbh_hi;    // (l * B + b) * H + h, absolute layer
-  int out_lo, out_hi;    // (l_rel * B + b) * H + h
-  int r0;                // first row of the chunk inside its segment
+  int nrows;         // < 0: this slot will get no more work
   int want_logits;
-  int nit;               // partials of this (l, b, h)
-  int item0_lo, item0_hi;  // first item of this (l, b)
-  int h;
+  long long glog;    // offset into p.logits of this chunk's first row
 };
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ long long join64(int lo, int hi) {
-  return (long long)(((unsigned long long)(unsigned)hi << 32) | (unsigned)lo);
+__device__ __forceinline__ unsigned fast_div(unsigned n, unsigned mul, unsigned shift) {
+  return (__umulhi(n, mul) + n) >> shift;  // exact for n < 2^31 (host: make_fast_div)
 }
 // Bounded wait of a whole warp that also gives up when another role has already aborted; the
 // answer is the same in every lane.
@@ -223,14 +246,13 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
   constexpr int RMAX = kTileBytes / ROWB;  // rows per item: 64 (128 for 128-byte rows)
   constexpr int TR = RMAX / kConsumers;    // rows per consumer warp
   constexpr int GR = TR / 8;               // groups of 8 rows per warp
-  constexpr int QD = D / 4;                // dims per lane
+  constexpr int DPL = D / 32;              // output dims per lane when a warp holds one vector
   constexpr int SLOTB = 2 * kTileBytes + kQBytes;
-  constexpr bool kDumpSplit = 32 * D > TR * ROWB;  // 8 x D floats do not fit a warp's K rows
-  static_assert(16 * D <= TR * ROWB, "warp result does not fit its own K and V rows");
+  static_assert(4 * D <= TR * ROWB, "a warp's result vector must fit its own K rows");
   static_assert(CPL >= 2 && CPL <= 8 && GR >= 1, "unsupported row size");
 
   extern __shared__ __align__(128) unsigned char smem[];
-  __shared__ __align__(8) uint64_t s_fullK[kSlots], s_fullV[kSlots], s_done[kSlots], s_empty[kSlots];
+  __shared__ __align__(8) uint64_t s_fullK[kSlots], s_fullV[kSlots], s_done[kSlots];
   __shared__ ItemDesc s_desc[kSlots];
   __shared__ float s_stat[kSlots][kConsumers][2];
   __shared__ int s_abort;
@@ -238,8 +260,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     for (int s = 0; s < kSlots; ++s) {
-      mbar_init(&s_fullK[s], 1); mbar_init(&s_fullV[s], 1);
-      mbar_init(&s_done[s], kConsumers); mbar_init(&s_empty[s], 1);
+      mbar_init(&s_fullK[s], 1); mbar_init(&s_fullV[s], 1); mbar_init(&s_done[s], kConsumers);
     }
     s_abort = 0;
     mbar_fence_init();
@@ -247,223 +268,201 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
   __syncthreads();
   volatile int* abort_flag = &s_abort;
   const int H = p.H;
-  const int total = p.total_work;
 
-  if (warp == 0) {
-    // ===================== producer =====================
-    int x_next = 0, end_marks = 0;
+  if (warp < kSlots) {
+    // ===================== manager of slot `warp` =====================
+    const int s = warp;
+    unsigned char* sK = smem + (size_t)s * SLOTB;
+    unsigned char* sV = sK + kTileBytes;
+    unsigned char* sQ = sV + kTileBytes;
+    const int total = p.total_work;
+    constexpr int VPR = ROWB / 16;            // 16-byte vectors per row
+    constexpr int LN = VPR <= 16 ? VPR : 16;  // lanes that carry one new row
+    constexpr int NV = VPR / LN;              // vectors per such lane
+
+    // A decoded work item, held in registers until its slot is free.
+    struct Dec {
+      bool valid, has_new;
+      int nrows, nbulk, want_logits;
+      long long slot, lbh, oidx, glog;
+      const unsigned char *srcK, *srcV;
+      T *newK, *newV;
+      uint4 nv[NV];
+    };
+    int lcur = 0;  // layer of the previous item: this warp's items arrive in increasing order
+    int x_next = 0;
     if (lane == 0) x_next = atomicAdd(p.work_counter, 1);
-    for (int round = 0;; ++round) {
-      const int s = round % kSlots;
-      const uint32_t par = (uint32_t)(round / kSlots) & 1u;
-      if (!ring_wait(&s_empty[s], par ^ 1u, abort_flag, p.status)) break;
+
+    auto decode = [&](Dec& d) {
       const int x = __shfl_sync(0xffffffffu, x_next, 0);
-      if (x >= total) {  // out of work: one end marker per slot, so that every merger sees one
-        if (lane == 0) { s_desc[s].nrows = -1; mbar_arrive(&s_fullK[s]); }
-        if (++end_marks == kSlots) break;
-        continue;
+      d.valid = x < total;
+      if (!d.valid) return;
+      if (lane == 0) x_next = atomicAdd(p.work_counter, 1);  // prefetch the index after this one
+      const int item = (int)fast_div((unsigned)x, p.h_mul, p.h_shift);
+      const int h = x - item * H;
+      while (lcur + 1 < p.layer_count && item >= p.lstart[lcur + 1]) ++lcur;
+      const int l_rel = lcur, l = p.layer_begin + l_rel;
+      const int cv = p.cvp[l_rel + 1] - p.cvp[l_rel];
+      const int per = cv + p.ct;
+      const int off = item - p.lstart[l_rel];
+      const int b = (int)fast_div((unsigned)off, p.per_mul[l_rel], p.per_shift[l_rel]);
+      const int c = off - b * per;
+      const bool is_vis = c < cv;
+      int seg_rows, rows_per, ci;
+      if (is_vis) {
+        seg_rows = p.ncur[l_rel]; rows_per = p.rpv[l_rel]; ci = c;
+      } else {
+        seg_rows = p.sys_len + __ldg(p.text_len + b) + p.step; rows_per = (seg_rows + p.ct - 1) / p.ct; ci = c - cv;
       }
-      if (lane == 0) x_next = atomicAdd(p.work_counter, 1);  // prefetch the next item index
-      const int h = x % H, item = x / H;
-      const Item it = decode_item(p, item);
-      const int l = p.layer_begin + it.l_rel, b = it.b;
-      const bool is_vis = it.c < it.cv;
-      int seg_rows, nchunk, ci;
-      if (is_vis) { seg_rows = p.ncur[it.l_rel]; nchunk = it.cv; ci = it.c; }
-      else { seg_rows = p.sys_len + __ldg(p.text_len + b) + p.step; nchunk = p.ct; ci = it.c - it.cv; }
-      const int rows_per = (seg_rows + nchunk - 1) / nchunk;
       const int r0 = ci * rows_per;
       int nrows = min(seg_rows, r0 + rows_per) - r0;
       if (nrows < 0) nrows = 0;
       if (nrows > RMAX) { nrows = RMAX; if (lane == 0) atomicOr(p.status, ST3_DEV_RANGE); }
-      const bool has_new = !is_vis && p.append && nrows > 0 && r0 + nrows == seg_rows;
-      const int nbulk = nrows - (has_new ? 1 : 0);
-      const long long lbh = ((long long)l * p.B + b) * H + h;
-      const long long oidx = ((long long)it.l_rel * p.B + b) * H + h;
-      T* blk = reinterpret_cast<T*>(p.cache) + lbh * p.lbh_stride;
+      d.has_new = !is_vis && p.append && nrows > 0 && r0 + nrows == seg_rows;
+      d.nrows = nrows;
+      d.nbulk = nrows - (d.has_new ? 1 : 0);
+      d.lbh = ((long long)l * p.B + b) * H + h;
+      d.oidx = ((long long)l_rel * p.B + b) * H + h;
+      T* blk = reinterpret_cast<T*>(p.cache) + d.lbh * p.lbh_stride;
       T* gK = is_vis ? blk : blk + 2LL * p.Nv * D;
       T* gV = gK + (is_vis ? (long long)p.Nv * D : (long long)p.cap_txt * D);
-      unsigned char* sK = smem + (size_t)s * SLOTB;
-      unsigned char* sV = sK + kTileBytes;
-      unsigned char* sQ = sV + kTileBytes;
-      if (has_new && lane < 2 * (ROWB / 16 <= 16 ? ROWB / 16 : 16)) {
-        // newest row: from the step's inputs to the cache and into the tile (ROWB/16 vectors each)
-        constexpr int VPR = ROWB / 16;
-        constexpr int LN = VPR <= 16 ? VPR : 16;
-        const int kv = lane / LN, c0 = lane % LN;
-        const T* src = reinterpret_cast<const T*>(kv ? p.v_new : p.k_new) + oidx * D;
-        T* dstg = (kv ? gV : gK) + (long long)(seg_rows - 1) * D;
-        for (int c = c0; c < VPR; c += LN) {
-          const uint4 val = __ldg(reinterpret_cast<const uint4*>(src) + c);
-          reinterpret_cast<uint4*>(dstg)[c] = val;
-          *reinterpret_cast<uint4*>((kv ? sV : sK) + (size_t)(nrows - 1) * ROWB + c * 16) = val;
+      d.srcK = reinterpret_cast<const unsigned char*>(gK) + (size_t)r0 * ROWB;
+      d.srcV = reinterpret_cast<const unsigned char*>(gV) + (size_t)r0 * ROWB;
+      d.want_logits = is_vis && p.ntgt[l_rel] < p.ncur[l_rel];
+      d.glog = d.lbh * p.Nv + r0;
+      d.slot = (long long)item * H + h;
+      if (d.has_new) {
+        // newest row: fetched from the step's inputs now, stored when the slot is free
+        d.newK = gK + (long long)(seg_rows - 1) * D;
+        d.newV = gV + (long long)(seg_rows - 1) * D;
+        if (lane < 2 * LN) {
+          const T* src = reinterpret_cast<const T*>(lane / LN ? p.v_new : p.k_new) + d.oidx * D;
+#pragma unroll
+          for (int i = 0; i < NV; ++i) d.nv[i] = __ldg(reinterpret_cast<const uint4*>(src) + (lane % LN) + i * LN);
         }
       }
-      __syncwarp();
+    };
+    // Starts the copies of a decoded item into this (free) slot.
+    auto issue = [&](const Dec& d) {
+      if (d.has_new) {
+        if (lane < 2 * LN) {
+          const int kv = lane / LN;
+#pragma unroll
+          for (int i = 0; i < NV; ++i) {
+            const int cc = (lane % LN) + i * LN;
+            reinterpret_cast<uint4*>(kv ? d.newV : d.newK)[cc] = d.nv[i];
+            *reinterpret_cast<uint4*>((kv ? sV : sK) + (size_t)(d.nrows - 1) * ROWB + cc * 16) = d.nv[i];
+          }
+        }
+        __syncwarp();
+      }
       if (lane == 0) {
-        ItemDesc& d = s_desc[s];
-        const long long slot = (long long)item * H + h;
-        const long long item0 = (long long)p.B * (p.cvp[it.l_rel] + it.l_rel * p.ct) + (long long)b * (it.cv + p.ct);
-        d.nrows = nrows;
-        d.slot_lo = (int)slot; d.slot_hi = (int)(slot >> 32);
-        d.lbh_lo = (int)lbh; d.lbh_hi = (int)(lbh >> 32);
-        d.out_lo = (int)oidx; d.out_hi = (int)(oidx >> 32);
-        d.r0 = r0;
-        d.want_logits = is_vis && p.ntgt[it.l_rel] < p.ncur[it.l_rel];
-        d.nit = it.cv + p.ct;
-        d.item0_lo = (int)item0; d.item0_hi = (int)(item0 >> 32);
-        d.h = h;
-        const uint32_t kb = (uint32_t)nbulk * ROWB;
+        ItemDesc& sd = s_desc[s];
+        sd.nrows = d.nrows; sd.want_logits = d.want_logits; sd.glog = d.glog;
+        const uint32_t kb = (uint32_t)d.nbulk * ROWB;
         mbar_expect_tx(&s_fullK[s], kb + ROWB);  // K rows + the query (D elements = ROWB bytes)
-        bulk_g2s(sQ, reinterpret_cast<const T*>(p.q) + oidx * D, ROWB, &s_fullK[s]);
-        if (kb) bulk_g2s(sK, reinterpret_cast<const unsigned char*>(gK) + (size_t)r0 * ROWB, kb, &s_fullK[s]);
+        bulk_g2s(sQ, reinterpret_cast<const T*>(p.q) + d.oidx * D, ROWB, &s_fullK[s]);
         if (kb) {
+          bulk_g2s(sK, d.srcK, kb, &s_fullK[s]);
           mbar_expect_tx(&s_fullV[s], kb);
-          bulk_g2s(sV, reinterpret_cast<const unsigned char*>(gV) + (size_t)r0 * ROWB, kb, &s_fullV[s]);
+          bulk_g2s(sV, d.srcV, kb, &s_fullV[s]);
         } else {
           mbar_arrive(&s_fullV[s]);
         }
       }
-    }
-  } else if (warp <= kSlots) {
-    // ===================== mergers: warp 1 + s serves ring slot s =====================
-    constexpr int DPL = D / 32;  // output dims per lane
-    const int s = warp - 1;
-    for (int use = 0;; ++use) {
-      const uint32_t par = (uint32_t)use & 1u;
-      if (!ring_wait(&s_done[s], par, abort_flag, p.status)) break;
-      const ItemDesc d = s_desc[s];
-      if (d.nrows < 0) break;
-      const int nw = (d.nrows + TR - 1) / TR;
-      float M = -INFINITY;
-      for (int w = 0; w < nw; ++w) M = fmaxf(M, s_stat[s][w][0]);
-      float Lsum = 0.f, o[DPL];
+    };
+    Dec cur, nxt;
+    decode(cur);
+    if (cur.valid) issue(cur);
+    else if (lane == 0) { s_desc[s].nrows = -1; mbar_arrive(&s_fullK[s]); }
+    for (int use = 0; cur.valid; ++use) {
+      decode(nxt);  // in the shadow of this item's copies and of the consumers' work
+      // ---- wait for the consumers, fold their eight results ----
+      if (!ring_wait(&s_done[s], (uint32_t)use & 1u, abort_flag, p.status)) break;
+      const int nw = (cur.nrows + TR - 1) / TR;
+      const float mw = lane < nw ? s_stat[s][lane][0] : -INFINITY;
+      const float lw = lane < nw ? s_stat[s][lane][1] : 0.f;
+      const float M = warp_max(mw);
+      const float wgt = lane < nw ? fast_exp2(mw - M) : 0.f;
+      const float Lsum = warp_sum(lw * wgt);
+      float po[DPL];
 #pragma unroll
-      for (int j = 0; j < DPL; ++j) o[j] = 0.f;
-      const unsigned char* sK = smem + (size_t)s * SLOTB;
-      for (int w = 0; w < nw; ++w) {
-        const float wgt = fast_exp2(s_stat[s][w][0] - M);
-        Lsum = fmaf(s_stat[s][w][1], wgt, Lsum);
-        const float* dumpK = reinterpret_cast<const float*>(sK + (size_t)w * TR * ROWB);
-        const float* dumpV = reinterpret_cast<const float*>(sK + kTileBytes + (size_t)w * TR * ROWB);
-        float t[DPL];
+      for (int j = 0; j < DPL; ++j) po[j] = 0.f;
 #pragma unroll
-        for (int j = 0; j < DPL; ++j) t[j] = 0.f;
+      for (int w = 0; w < kConsumers; ++w) {
+        const float ww = __shfl_sync(0xffffffffu, wgt, w);
+        if (w < nw) {
+          const float* res = reinterpret_cast<const float*>(sK + (size_t)w * TR * ROWB) + lane * DPL;  // [D]
 #pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          const float* dump = kDumpSplit ? (g >= 4 ? dumpV - 4 * D : dumpK) : dumpK;
-          if (DPL == 4) {
-            const float4 v4 = *reinterpret_cast<const float4*>(dump + g * D + lane * 4);
-            t[0] += v4.x; t[1] += v4.y; t[2] += v4.z; t[DPL - 1] += v4.w;
-          } else {
-            const float2 v2 = *reinterpret_cast<const float2*>(dump + g * D + lane * 2);
-            t[0] += v2.x; t[DPL - 1] += v2.y;
+          for (int j = 0; j < DPL; j += 2) {
+            const float2 v2 = *reinterpret_cast<const float2*>(res + j);
+            po[j] = fmaf(v2.x, ww, po[j]); po[j + 1] = fmaf(v2.y, ww, po[j + 1]);
           }
         }
-#pragma unroll
-        for (int j = 0; j < DPL; ++j) o[j] = fmaf(t[j], wgt, o[j]);
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&s_empty[s]);  // the slot may be refilled from here on
-      const long long slot = join64(d.slot_lo, d.slot_hi);
-      if (d.nrows == 0) M = -INFINITY;
+      __syncwarp();  // every lane is done reading the slot before it is refilled
+      // ---- refill the slot at once ----
+      if (nxt.valid) issue(nxt);
+      else if (lane == 0) { s_desc[s].nrows = -1; mbar_arrive(&s_fullK[s]); }  // end marker
+      // ---- publish this item's partial (plain stores: the next kernel merges the partials) ----
 #pragma unroll
-      for (int j = 0; j < DPL; ++j) p.part_acc[slot * D + lane * DPL + j] = o[j];
-      if (lane == 0) { p.part_ml[2 * slot] = M; p.part_ml[2 * slot + 1] = Lsum; }
-      // ticket: whoever publishes the last partial of this (l, b, h) merges them all
-      __threadfence();
-      __syncwarp();
-      int last = 0;
-      const long long lbh = join64(d.lbh_lo, d.lbh_hi);
-      if (lane == 0) {
-        const int old = atomicAdd(p.tickets + lbh, 1);
-        last = (old == d.nit - 1);
-        if (last) p.tickets[lbh] = 0;  // ready for the next step
-      }
-      last = __shfl_sync(0xffffffffu, last, 0);
-      if (last) {
-        __threadfence();
-        const long long item0 = join64(d.item0_lo, d.item0_hi);
-        float Mh = -INFINITY;
-        for (int i = lane; i < d.nit; i += 32) Mh = fmaxf(Mh, __ldcg(p.part_ml + 2 * ((item0 + i) * H + d.h)));
-        Mh = warp_max(Mh);
-        float Lh = 0.f;
-        for (int i = lane; i < d.nit; i += 32) {
-          const long long sl = (item0 + i) * H + d.h;
-          Lh += __ldcg(p.part_ml + 2 * sl + 1) * fast_exp2(__ldcg(p.part_ml + 2 * sl) - Mh);
-        }
-        Lh = warp_sum(Lh);
-        float oh[DPL];
-#pragma unroll
-        for (int j = 0; j < DPL; ++j) oh[j] = 0.f;
-        for (int i = 0; i < d.nit; ++i) {
-          const long long sl = (item0 + i) * H + d.h;
-          const float wgt = fast_exp2(__ldcg(p.part_ml + 2 * sl) - Mh);
-#pragma unroll
-          for (int j = 0; j < DPL; ++j) oh[j] = fmaf(wgt, __ldcg(p.part_acc + sl * D + lane * DPL + j), oh[j]);
-        }
-        const float invL = 1.f / Lh;
-        T* out = reinterpret_cast<T*>(p.out) + join64(d.out_lo, d.out_hi) * D;
-#pragma unroll
-        for (int j = 0; j < DPL; ++j) store_out(out + lane * DPL + j, oh[j] * invL);
-        if (lane == 0) { p.head_stat[2 * lbh] = Mh; p.head_stat[2 * lbh + 1] = invL; }
-      }
+      for (int j = 0; j < DPL; ++j) p.part_acc[cur.slot * D + lane * DPL + j] = po[j];
+      if (lane == 0) { p.part_ml[2 * cur.slot] = M; p.part_ml[2 * cur.slot + 1] = Lsum; }
+      cur = nxt;
     }
   } else {
     // ===================== consumers =====================
-    const int w = warp - 1 - kSlots;
+    const int w = warp - kSlots;
     const int r8 = lane >> 2, c4 = lane & 3;
-    int rot, end_marks = 0;
+    int rot;
     if (CPL == 2) rot = r8 & 1;
     else if (CPL == 4) rot = (c4 >> 1) + 2 * (r8 & 1);
     else rot = lane & 7;
-    for (int round = 0;; ++round) {
+    const float sc = 1.4426950408889634f * rsqrtf((float)D);
+    unsigned live = (1u << kSlots) - 1;  // slots that may still deliver work
+    for (int round = 0; live; ++round) {
       const int s = round % kSlots;
+      if (!(live & (1u << s))) continue;
       const uint32_t par = (uint32_t)(round / kSlots) & 1u;
       if (!ring_wait(&s_fullK[s], par, abort_flag, p.status)) break;
       const int nrows = s_desc[s].nrows;
-      if (nrows < 0) {  // end marker: pass it on to this slot's merger; the last one ends the warp
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&s_done[s]);
-        if (++end_marks == kSlots) break;
-        continue;
-      }
+      if (nrows < 0) { live &= ~(1u << s); continue; }
       const int base = w * TR;
       if (base < nrows) {
         unsigned char* sK = smem + (size_t)s * SLOTB;
         const unsigned char* sV = sK + kTileBytes;
         const unsigned char* sQ = sV + kTileBytes;
-        const float sc = 1.4426950408889634f * rsqrtf((float)D);
         // this lane's quarter of the query, in the rotated chunk order it reads rows in
-        float qf[CPL][EPL];
+        u64 q2[CPL][EPL / 2];
 #pragma unroll
         for (int j = 0; j < CPL; ++j) {
           const int jj = (j + rot) & (CPL - 1);
-          unpack16(*reinterpret_cast<const uint4*>(sQ + (c4 * CPL + jj) * 16), qf[j]);
+          unpack16_pairs(*reinterpret_cast<const uint4*>(sQ + (c4 * CPL + jj) * 16), q2[j]);
         }
+        // ---- K pass: four lanes per row, one logit per row ----
         float sl[GR];
         bool ok[GR];
 #pragma unroll
         for (int g = 0; g < GR; ++g) {
           const int r = base + g * 8 + r8;
           ok[g] = r < nrows;
-          float a[CPL];
+          u64 a2[CPL];
 #pragma unroll
-          for (int j = 0; j < CPL; ++j) a[j] = 0.f;
+          for (int j = 0; j < CPL; ++j) a2[j] = 0ull;
           if (ok[g]) {
             const unsigned char* row = sK + (size_t)r * ROWB + c4 * (CPL * 16);
 #pragma unroll
             for (int j = 0; j < CPL; ++j) {
               const int jj = (j + rot) & (CPL - 1);
-              float kf[EPL];
-              unpack16(*reinterpret_cast<const uint4*>(row + jj * 16), kf);
+              u64 k2[EPL / 2];
+              unpack16_pairs(*reinterpret_cast<const uint4*>(row + jj * 16), k2);
 #pragma unroll
-              for (int e = 0; e < EPL; ++e) a[j] = fmaf(qf[j][e], kf[e], a[j]);
+              for (int e = 0; e < EPL / 2; ++e) fma2(a2[j], q2[j][e], k2[e]);
             }
           }
           float t = 0.f;
 #pragma unroll
-          for (int j = 0; j < CPL; ++j) t += a[j];
+          for (int j = 0; j < CPL; ++j) t += sum2(a2[j]);
           t += __shfl_xor_sync(0xffffffffu, t, 1);
           t += __shfl_xor_sync(0xffffffffu, t, 2);
           sl[g] = ok[g] ? t * sc : -INFINITY;  // log2-domain logit
@@ -472,9 +471,8 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
 #pragma unroll
         for (int g = 1; g < GR; ++g) m = fmaxf(m, sl[g]);
         m = warp_max(m);
-        const ItemDesc& d = s_desc[s];
-        if (d.want_logits && c4 == 0) {
-          float* glog = p.logits + join64(d.lbh_lo, d.lbh_hi) * p.Nv + d.r0;
+        if (s_desc[s].want_logits && c4 == 0) {
+          float* glog = p.logits + s_desc[s].glog;
 #pragma unroll
           for (int g = 0; g < GR; ++g)
             if (ok[g]) glog[base + g * 8 + r8] = sl[g];
@@ -487,37 +485,30 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
         }
         lsum = warp_sum(lsum);
         if (!ring_wait(&s_fullV[s], par, abort_flag, p.status)) break;
-        float acc[CPL][EPL];
+        // ---- V pass: a lane owns DPL output dims and walks this warp's rows ----
+        const int nmine = min(TR, nrows - base);
+        u64 acc2[DPL / 2];
 #pragma unroll
-        for (int j = 0; j < CPL; ++j)
+        for (int i = 0; i < DPL / 2; ++i) acc2[i] = 0ull;
+        const unsigned char* vrow = sV + (size_t)base * ROWB + lane * (DPL * (int)sizeof(T));
 #pragma unroll
-          for (int e = 0; e < EPL; ++e) acc[j][e] = 0.f;
+        for (int rr = 0; rr < TR; ++rr) {
+          const float pv = __shfl_sync(0xffffffffu, pr[rr / 8], (rr % 8) * 4);
+          if (rr < nmine) {
+            u64 v2[DPL / 2];
+            load_pairs<T, DPL>(vrow + (size_t)rr * ROWB, v2);
+            const u64 pp = pack2(pv, pv);
 #pragma unroll
-        for (int g = 0; g < GR; ++g) {
-          if (ok[g]) {
-            const unsigned char* row = sV + (size_t)(base + g * 8 + r8) * ROWB + c4 * (CPL * 16);
-#pragma unroll
-            for (int j = 0; j < CPL; ++j) {
-              const int jj = (j + rot) & (CPL - 1);
-              float vf[EPL];
-              unpack16(*reinterpret_cast<const uint4*>(row + jj * 16), vf);
-#pragma unroll
-              for (int e = 0; e < EPL; ++e) acc[j][e] = fmaf(pr[g], vf[e], acc[j][e]);
-            }
+            for (int i = 0; i < DPL / 2; ++i) fma2(acc2[i], pp, v2[i]);
           }
         }
-        // dump [8 row groups][D] over this warp's own K rows (and, where those are too small, half of
-        // it over its own V rows)
-        __syncwarp();  // every lane has finished reading this warp's V rows as well
-        float* dump = reinterpret_cast<float*>((kDumpSplit && r8 >= 4 ? sK + kTileBytes : sK) + (size_t)base * ROWB) +
-                      (kDumpSplit ? (r8 & 3) : r8) * D + c4 * QD;
+        // the warp's un-normalised result [D] goes over its own (consumed) K rows
+        float* res = reinterpret_cast<float*>(sK + (size_t)base * ROWB) + lane * DPL;
 #pragma unroll
-        for (int j = 0; j < CPL; ++j) {
-          const int jj = (j + rot) & (CPL - 1);
-#pragma unroll
-          for (int e = 0; e < EPL; e += 4)
-            *reinterpret_cast<float4*>(dump + jj * EPL + e) =
-                make_float4(acc[j][e], acc[j][e + 1], acc[j][e + 2], acc[j][e + 3]);
+        for (int i = 0; i < DPL / 2; ++i) {
+          float lo, hi;
+          split2(acc2[i], lo, hi);
+          *reinterpret_cast<float2*>(res + 2 * i) = make_float2(lo, hi);
         }
         if (lane == 0) { s_stat[s][w][0] = m; s_stat[s][w][1] = lsum; }
       }
@@ -531,14 +522,14 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
 // Merge partials, visual scores, top-k (Eq. 3), in-place compaction (Eq. 7's eviction)
 // ------------------------------------------------------------------------------------------
 template <typename T, int D>
-__global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p) {
+__global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepParams p) {
   constexpr int ROWB = D * sizeof(T);
   constexpr int VPR = ROWB / 16;  // 16-byte vectors per row
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ float s_M[kMaxHeads];
   __shared__ float s_invL[kMaxHeads];
   __shared__ int s_hist[256];
-  __shared__ int s_scan[kWarps];
+  __shared__ int s_scan[kFinishWarps];
   __shared__ int s_sel[3];  // digit, count above, count in bin
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -546,6 +537,39 @@ __global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p
   const int l_rel = blockIdx.x / B, b = blockIdx.x % B;
   const int l = p.layer_begin + l_rel;
   if (blockIdx.x == 0 && tid == 0) *p.work_counter = 0;  // the next attention launch starts from item 0
+
+  // ---- merge the chunk partials of every head (one warp per head) ----
+  {
+    const int nit = p.cvp[l_rel + 1] - p.cvp[l_rel] + p.ct;
+    const long long item0 = (long long)p.lstart[l_rel] + (long long)b * nit;
+    constexpr int DPL = D / 32;
+    for (int h = warp; h < H; h += kFinishWarps) {
+      float M = -INFINITY;
+      for (int i = lane; i < nit; i += 32) M = fmaxf(M, p.part_ml[2 * ((item0 + i) * H + h)]);
+      M = warp_max(M);
+      float Lh = 0.f;
+      for (int i = lane; i < nit; i += 32) {
+        const long long sl = (item0 + i) * H + h;
+        Lh += p.part_ml[2 * sl + 1] * fast_exp2(p.part_ml[2 * sl] - M);
+      }
+      Lh = warp_sum(Lh);
+      float o[DPL];
+#pragma unroll
+      for (int j = 0; j < DPL; ++j) o[j] = 0.f;
+      for (int i = 0; i < nit; ++i) {
+        const long long sl = (item0 + i) * H + h;
+        const float wgt = fast_exp2(p.part_ml[2 * sl] - M);
+#pragma unroll
+        for (int j = 0; j < DPL; ++j) o[j] = fmaf(wgt, p.part_acc[sl * D + lane * DPL + j], o[j]);
+      }
+      const float invL = 1.f / Lh;
+      T* out = reinterpret_cast<T*>(p.out) + (((long long)l_rel * B + b) * H + h) * D;
+#pragma unroll
+      for (int j = 0; j < DPL; ++j) store_out(out + lane * DPL + j, o[j] * invL);
+      if (lane == 0) { s_M[h] = M; s_invL[h] = invL; }
+    }
+  }
+  __syncthreads();
   const long long lb = (long long)l * B + b;
   const int n_cur = p.n_cur[lb];
   if (n_cur != p.ncur[l_rel]) {  // host bookkeeping and device state disagree: flag, do not touch
@@ -561,15 +585,9 @@ __global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p
   int* ids = p.ids + lb * Nv;
   float* mass_by_id = p.mass_by_id + lb * Nv;
 
-  for (int h = tid; h < H; h += kThreads) {
-    s_M[h] = p.head_stat[2 * (lb * H + h)];
-    s_invL[h] = p.head_stat[2 * (lb * H + h) + 1];
-  }
-  __syncthreads();
-
   // ---- visual scores: probability of every visual row summed over heads ----
   bool bad = false;
-  for (int i = tid; i < n_cur; i += kThreads) {
+  for (int i = tid; i < n_cur; i += kFinishThreads) {
     float mass = 0.f;
     const float* lg = p.logits + lb * H * Nv + i;
     for (int h = 0; h < H; ++h) mass += fast_exp2(lg[(long long)h * Nv] - s_M[h]) * s_invL[h];
@@ -586,9 +604,9 @@ __global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p
   if (k > 0) {
     int need = k;
     for (int shift = 56; shift >= 0; shift -= 8) {
-      s_hist[tid] = 0;
+      if (tid < 256) s_hist[tid] = 0;
       __syncthreads();
-      for (int i = tid; i < n_cur; i += kThreads) {
+      for (int i = tid; i < n_cur; i += kFinishThreads) {
         const unsigned long long key = s_key[i];
         if ((key & mask) == prefix) atomicAdd(&s_hist[(int)((key >> shift) & 0xffull)], 1);
       }
@@ -624,7 +642,7 @@ __global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p
   }
 
   // ---- pair every hole among the first k rows with a kept row of the tail ----
-  const int per = (n_cur + kThreads - 1) / kThreads;
+  const int per = (n_cur + kFinishThreads - 1) / kFinishThreads;
   const int i0 = min(n_cur, tid * per), i1 = min(n_cur, i0 + per);
   int nh = 0, nm = 0;
   for (int i = i0; i < i1; ++i) {
@@ -643,7 +661,7 @@ __global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p
   __syncthreads();
   int woff = 0, total = 0;
 #pragma unroll
-  for (int w = 0; w < kWarps; ++w) {
+  for (int w = 0; w < kFinishWarps; ++w) {
     if (w < warp) woff += s_scan[w];
     total += s_scan[w];
   }
@@ -664,7 +682,7 @@ __global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p
   // ---- move the rows (sources are rows >= k, destinations rows < k: disjoint) ----
   unsigned char* blk0 = reinterpret_cast<unsigned char*>(p.cache) + (size_t)(lb * H) * p.lbh_stride * sizeof(T);
   const long long nvec = (long long)nmove * H * 2 * VPR;
-  for (long long v = tid; v < nvec; v += kThreads) {
+  for (long long v = tid; v < nvec; v += kFinishThreads) {
     const int c = (int)(v % VPR);
     long long r = v / VPR;
     const int kv = (int)(r % 2); r /= 2;
@@ -674,7 +692,7 @@ __global__ void __launch_bounds__(kThreads) st3_finish_kernel(const StepParams p
     const uint4 val = *reinterpret_cast<const uint4*>(base + (size_t)s_mover[j] * ROWB + c * 16);
     *reinterpret_cast<uint4*>(base + (size_t)s_hole[j] * ROWB + c * 16) = val;
   }
-  for (int j = tid; j < nmove; j += kThreads) ids[s_hole[j]] = ids[s_mover[j]];
+  for (int j = tid; j < nmove; j += kFinishThreads) ids[s_hole[j]] = ids[s_mover[j]];
   if (tid == 0) p.n_cur[lb] = k;
 }
 
@@ -725,10 +743,17 @@ __global__ void __launch_bounds__(kThreads) st3_ingest_kernel(const StepParams p
 // Host side
 // ------------------------------------------------------------------------------------------
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+// n / d == (umulhi(n, mul) + n) >> shift for every n < 2^31 (division by an invariant integer).
+inline void make_fast_div(unsigned d, unsigned* mul, unsigned* shift) {
+  unsigned L = 0;
+  while ((1ull << L) < d) ++L;
+  *mul = (unsigned)((((1ull << 32) * ((1ull << L) - d)) / d) + 1);
+  *shift = L;
+}
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 struct Layout {
-  size_t elem, cache, part_ml, part_acc, logits, mass, ids, n_cur, tickets, head_stat, text_len, status, stage_q, stage_k, stage_v,
+  size_t elem, cache, part_ml, part_acc, logits, mass, ids, n_cur, text_len, status, stage_q, stage_k, stage_v,
       stage_o, total;
   long long lbh_stride;
   int cap_txt, chunk_rows, max_items;
@@ -786,8 +811,6 @@ Layout make_layout(const st3_config* c) {
   L.mass = take(lb * (size_t)c->num_visual * sizeof(float));
   L.ids = take(lb * (size_t)c->num_visual * sizeof(int));
   L.n_cur = take(lb * sizeof(int));
-  L.tickets = take(lbh * sizeof(int));
-  L.head_stat = take(lbh * 2 * sizeof(float));
   L.text_len = take((size_t)c->batch * sizeof(int));
   L.status = take(256);
   const size_t io = lbh * c->head_dim * L.elem;
@@ -863,7 +886,7 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
   (void)total_items;
   st3_attend_kernel<T, D><<<(unsigned)(ctx->num_sms * ctx->attend_ctas_per_sm), kAttendThreads, ctx->attend_smem, st>>>(p);
   if (e1) cudaEventRecord(e1, st);
-  st3_finish_kernel<T, D><<<(unsigned)(p.layer_count * c.batch), kThreads, ctx->finish_smem, st>>>(p);
+  st3_finish_kernel<T, D><<<(unsigned)(p.layer_count * c.batch), kFinishThreads, ctx->finish_smem, st>>>(p);
   if (e2) cudaEventRecord(e2, st);
   ctx->launches += 2;
   return cudaGetLastError() == cudaSuccess ? ST3_OK : ST3_ERR_CUDA;
@@ -905,8 +928,6 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
   p.text_len = reinterpret_cast<const int*>(ctx->ws + L.text_len);
   p.status = reinterpret_cast<int*>(ctx->ws + L.status);
   p.work_counter = p.status + 16;
-  p.tickets = reinterpret_cast<int*>(ctx->ws + L.tickets);
-  p.head_stat = reinterpret_cast<float*>(ctx->ws + L.head_stat);
   p.lbh_stride = L.lbh_stride;
   p.layer_begin = layer_begin; p.layer_count = layer_count; p.B = c.batch; p.H = c.num_heads;
   p.sys_len = c.sys_len; p.Nv = c.num_visual; p.cap_txt = L.cap_txt; p.step = step; p.append = prefill ? 0 : 1;
@@ -920,8 +941,14 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
     const int tgt = ctx->n_tab[(size_t)l * (c.max_decode_steps + 1) + step];
     p.ncur[i] = ncur;
     p.ntgt[i] = tgt < ncur ? tgt : ncur;
-    p.cvp[i + 1] = p.cvp[i] + ceil_div(ncur, R);
+    const int cv = ceil_div(ncur, R);
+    p.cvp[i + 1] = p.cvp[i] + cv;
+    p.lstart[i] = c.batch * (p.cvp[i] + i * p.ct);
+    p.rpv[i] = cv ? ceil_div(ncur, cv) : 0;
+    make_fast_div((unsigned)(cv + p.ct), &p.per_mul[i], &p.per_shift[i]);
   }
+  p.lstart[layer_count] = c.batch * (p.cvp[layer_count] + layer_count * p.ct);
+  make_fast_div((unsigned)c.num_heads, &p.h_mul, &p.h_shift);
   const long long total_items = (long long)c.batch * (p.cvp[layer_count] + (long long)layer_count * p.ct);
   if (total_items > L.max_items || total_items * c.num_heads > 0x3fffffffLL) return ST3_ERR_CAPACITY;
   p.total_work = (int)(total_items * c.num_heads);

@@ -196,13 +196,16 @@ __device__ __forceinline__ float warp_sum(float v) {
 // the item's K rows, V rows and query into its slot with bulk asynchronous copies, and - once the
 // consumers are done with the slot - folds their eight results into the item's partial, refills
 // the slot at once and only then stores the partial (plain stores; st3_finish_kernel merges the
-// partials of each head).  Warps 3..10 are CONSUMERS: each owns a fixed 1/8 of an item's rows
+// partials of each head).  Warps 3..10 are CONSUMERS in two groups of four that take the slot
+// uses alternately (so two items are always being computed); a warp owns a fixed 1/4 of an item's rows
 // (K pass: four lanes per row; V pass: a lane owns D/32 output dims and walks the warp's rows):
 // logits, tile-local softmax, p.V; the warp leaves its un-normalised result over its own,
 // already consumed, K rows.  Loads of the other slots
 // are always in flight while one slot is being computed.  Every mbarrier wait is bounded; a
 // timeout raises a block-wide abort flag that ends all roles.
 constexpr int kConsumers = 8;
+constexpr int kGroups = 2;  // consumer warps work in two groups, on two ring slots at a time
+constexpr int kGroupWarps = kConsumers / kGroups;
 constexpr int kSlots = 3;
 constexpr int kAttendThreads = 32 * (kSlots + kConsumers);
 constexpr int kQBytes = 512;
@@ -244,7 +247,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
   constexpr int CPL = ROWB / 64;           // 16-byte chunks per lane (a lane owns a quarter row)
   constexpr int kTileBytes = ROWB >= 512 ? 32768 : 16384;  // K (and V) bytes of one ring slot
   constexpr int RMAX = kTileBytes / ROWB;  // rows per item: 64 (128 for 128-byte rows)
-  constexpr int TR = RMAX / kConsumers;    // rows per consumer warp
+  constexpr int TR = RMAX / kGroupWarps;   // rows per consumer warp
   constexpr int GR = TR / 8;               // groups of 8 rows per warp
   constexpr int DPL = D / 32;              // output dims per lane when a warp holds one vector
   constexpr int SLOTB = 2 * kTileBytes + kQBytes;
@@ -252,16 +255,19 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
   static_assert(CPL >= 2 && CPL <= 8 && GR >= 1, "unsupported row size");
 
   extern __shared__ __align__(128) unsigned char smem[];
-  __shared__ __align__(8) uint64_t s_fullK[kSlots], s_fullV[kSlots], s_done[kSlots];
+  // one barrier set per (slot, consumer group): a group sees every phase of its own barriers, so
+  // phase parity is never ambiguous
+  __shared__ __align__(8) uint64_t s_fullK[kSlots][kGroups], s_fullV[kSlots][kGroups], s_done[kSlots][kGroups];
   __shared__ ItemDesc s_desc[kSlots];
-  __shared__ float s_stat[kSlots][kConsumers][2];
+  __shared__ float s_stat[kSlots][kGroupWarps][2];
   __shared__ int s_abort;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
-    for (int s = 0; s < kSlots; ++s) {
-      mbar_init(&s_fullK[s], 1); mbar_init(&s_fullV[s], 1); mbar_init(&s_done[s], kConsumers);
-    }
+    for (int s = 0; s < kSlots; ++s)
+      for (int g = 0; g < kGroups; ++g) {
+        mbar_init(&s_fullK[s][g], 1); mbar_init(&s_fullV[s][g], 1); mbar_init(&s_done[s][g], kGroupWarps);
+      }
     s_abort = 0;
     mbar_fence_init();
   }
@@ -343,7 +349,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
       }
     };
     // Starts the copies of a decoded item into this (free) slot.
-    auto issue = [&](const Dec& d) {
+    auto issue = [&](const Dec& d, int g) {  // g: the consumer group this use of the slot belongs to
       if (d.has_new) {
         if (lane < 2 * LN) {
           const int kv = lane / LN;
@@ -360,25 +366,26 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
         ItemDesc& sd = s_desc[s];
         sd.nrows = d.nrows; sd.want_logits = d.want_logits; sd.glog = d.glog;
         const uint32_t kb = (uint32_t)d.nbulk * ROWB;
-        mbar_expect_tx(&s_fullK[s], kb + ROWB);  // K rows + the query (D elements = ROWB bytes)
-        bulk_g2s(sQ, reinterpret_cast<const T*>(p.q) + d.oidx * D, ROWB, &s_fullK[s]);
+        mbar_expect_tx(&s_fullK[s][g], kb + ROWB);  // K rows + the query (D elements = ROWB bytes)
+        bulk_g2s(sQ, reinterpret_cast<const T*>(p.q) + d.oidx * D, ROWB, &s_fullK[s][g]);
         if (kb) {
-          bulk_g2s(sK, d.srcK, kb, &s_fullK[s]);
-          mbar_expect_tx(&s_fullV[s], kb);
-          bulk_g2s(sV, d.srcV, kb, &s_fullV[s]);
+          bulk_g2s(sK, d.srcK, kb, &s_fullK[s][g]);
+          mbar_expect_tx(&s_fullV[s][g], kb);
+          bulk_g2s(sV, d.srcV, kb, &s_fullV[s][g]);
         } else {
-          mbar_arrive(&s_fullV[s]);
+          mbar_arrive(&s_fullV[s][g]);
         }
       }
     };
     Dec cur, nxt;
     decode(cur);
-    if (cur.valid) issue(cur);
-    else if (lane == 0) { s_desc[s].nrows = -1; mbar_arrive(&s_fullK[s]); }
+    // Use u of this slot belongs to consumer group (u + s) % kGroups and is that group's (u / kGroups)-th
+    // use of the slot, which fixes the parity of the group's barriers.
+    if (cur.valid) issue(cur, s % kGroups);
     for (int use = 0; cur.valid; ++use) {
       decode(nxt);  // in the shadow of this item's copies and of the consumers' work
-      // ---- wait for the consumers, fold their eight results ----
-      if (!ring_wait(&s_done[s], (uint32_t)use & 1u, abort_flag, p.status)) break;
+      // ---- wait for this use's consumer group, fold its warps' results ----
+      if (!ring_wait(&s_done[s][(use + s) % kGroups], (uint32_t)(use / kGroups) & 1u, abort_flag, p.status)) break;
       const int nw = (cur.nrows + TR - 1) / TR;
       const float mw = lane < nw ? s_stat[s][lane][0] : -INFINITY;
       const float lw = lane < nw ? s_stat[s][lane][1] : 0.f;
@@ -389,7 +396,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
 #pragma unroll
       for (int j = 0; j < DPL; ++j) po[j] = 0.f;
 #pragma unroll
-      for (int w = 0; w < kConsumers; ++w) {
+      for (int w = 0; w < kGroupWarps; ++w) {
         const float ww = __shfl_sync(0xffffffffu, wgt, w);
         if (w < nw) {
           const float* res = reinterpret_cast<const float*>(sK + (size_t)w * TR * ROWB) + lane * DPL;  // [D]
@@ -402,17 +409,22 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
       }
       __syncwarp();  // every lane is done reading the slot before it is refilled
       // ---- refill the slot at once ----
-      if (nxt.valid) issue(nxt);
-      else if (lane == 0) { s_desc[s].nrows = -1; mbar_arrive(&s_fullK[s]); }  // end marker
+      if (nxt.valid) issue(nxt, (use + 1 + s) % kGroups);
       // ---- publish this item's partial (plain stores: the next kernel merges the partials) ----
 #pragma unroll
       for (int j = 0; j < DPL; ++j) p.part_acc[cur.slot * D + lane * DPL + j] = po[j];
       if (lane == 0) { p.part_ml[2 * cur.slot] = M; p.part_ml[2 * cur.slot + 1] = Lsum; }
       cur = nxt;
     }
+    // out of work (or aborted): an end marker for each consumer group, on the group's own barrier
+    if (lane == 0) {
+      s_desc[s].nrows = -1;
+      for (int g = 0; g < kGroups; ++g) mbar_arrive(&s_fullK[s][g]);
+    }
   } else {
     // ===================== consumers =====================
-    const int w = warp - kSlots;
+    const int grp = (warp - kSlots) / kGroupWarps;
+    const int w = (warp - kSlots) % kGroupWarps;
     const int r8 = lane >> 2, c4 = lane & 3;
     int rot;
     if (CPL == 2) rot = r8 & 1;
@@ -422,9 +434,10 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
     unsigned live = (1u << kSlots) - 1;  // slots that may still deliver work
     for (int round = 0; live; ++round) {
       const int s = round % kSlots;
-      if (!(live & (1u << s))) continue;
-      const uint32_t par = (uint32_t)(round / kSlots) & 1u;
-      if (!ring_wait(&s_fullK[s], par, abort_flag, p.status)) break;
+      const int use = round / kSlots;  // round r is use r / kSlots of slot r % kSlots
+      if ((use + s) % kGroups != grp || !(live & (1u << s))) continue;
+      const uint32_t par = (uint32_t)(use / kGroups) & 1u;
+      if (!ring_wait(&s_fullK[s][grp], par, abort_flag, p.status)) break;
       const int nrows = s_desc[s].nrows;
       if (nrows < 0) { live &= ~(1u << s); continue; }
       const int base = w * TR;
@@ -484,7 +497,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
           if (c4 == 0) lsum += pr[g];
         }
         lsum = warp_sum(lsum);
-        if (!ring_wait(&s_fullV[s], par, abort_flag, p.status)) break;
+        if (!ring_wait(&s_fullV[s][grp], par, abort_flag, p.status)) break;
         // ---- V pass: a lane owns DPL output dims and walks this warp's rows ----
         const int nmine = min(TR, nrows - base);
         u64 acc2[DPL / 2];
@@ -513,7 +526,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
         if (lane == 0) { s_stat[s][w][0] = m; s_stat[s][w][1] = lsum; }
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(&s_done[s]);
+      if (lane == 0) mbar_arrive(&s_done[s][grp]);
     }
   }
 }

@@ -544,6 +544,7 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   __shared__ int s_hist[256];
   __shared__ int s_scan[kFinishWarps];
   __shared__ int s_sel[3];  // digit, count above, count in bin
+  __shared__ float s_half[kFinishThreads / 2];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int B = p.B, H = p.H, Nv = p.Nv;
@@ -551,29 +552,57 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   const int l = p.layer_begin + l_rel;
   if (blockIdx.x == 0 && tid == 0) *p.work_counter = 0;  // the next attention launch starts from item 0
 
+  const long long lb = (long long)l * B + b;
+  const int n_dev = p.n_cur[lb];  // needed only after the merge: the load overlaps it
+
   // ---- merge the chunk partials of every head (one warp per head) ----
+  // Loads are issued in batches so that a head costs one memory round trip per kMergeBatch partials.
   {
+    constexpr int DPL = D / 32;
+    constexpr int kMergeBatch = 8;
     const int nit = p.cvp[l_rel + 1] - p.cvp[l_rel] + p.ct;
     const long long item0 = (long long)p.lstart[l_rel] + (long long)b * nit;
-    constexpr int DPL = D / 32;
+    const float2* ml = reinterpret_cast<const float2*>(p.part_ml);
     for (int h = warp; h < H; h += kFinishWarps) {
+      float a[kMergeBatch][DPL];
+      auto load_batch = [&](int i0) {
+#pragma unroll
+        for (int i = 0; i < kMergeBatch; ++i) {
+          if (i0 + i < nit) {
+            const float* src = p.part_acc + ((item0 + i0 + i) * H + h) * D + lane * DPL;
+            if (DPL == 4) {
+              const float4 v = *reinterpret_cast<const float4*>(src);
+              a[i][0] = v.x; a[i][1] = v.y; a[i][DPL - 2] = v.z; a[i][DPL - 1] = v.w;
+            } else {
+              const float2 v = *reinterpret_cast<const float2*>(src);
+              a[i][0] = v.x; a[i][DPL - 1] = v.y;
+            }
+          }
+        }
+      };
+      load_batch(0);
       float M = -INFINITY;
-      for (int i = lane; i < nit; i += 32) M = fmaxf(M, p.part_ml[2 * ((item0 + i) * H + h)]);
+      for (int i = lane; i < nit; i += 32) M = fmaxf(M, ml[(item0 + i) * H + h].x);
       M = warp_max(M);
       float Lh = 0.f;
       for (int i = lane; i < nit; i += 32) {
-        const long long sl = (item0 + i) * H + h;
-        Lh += p.part_ml[2 * sl + 1] * fast_exp2(p.part_ml[2 * sl] - M);
+        const float2 v = ml[(item0 + i) * H + h];
+        Lh += v.y * fast_exp2(v.x - M);
       }
       Lh = warp_sum(Lh);
       float o[DPL];
 #pragma unroll
       for (int j = 0; j < DPL; ++j) o[j] = 0.f;
-      for (int i = 0; i < nit; ++i) {
-        const long long sl = (item0 + i) * H + h;
-        const float wgt = fast_exp2(p.part_ml[2 * sl] - M);
+      for (int i0 = 0; i0 < nit; i0 += kMergeBatch) {
+        if (i0) load_batch(i0);
 #pragma unroll
-        for (int j = 0; j < DPL; ++j) o[j] = fmaf(wgt, p.part_acc[sl * D + lane * DPL + j], o[j]);
+        for (int i = 0; i < kMergeBatch; ++i) {
+          if (i0 + i < nit) {
+            const float wgt = fast_exp2(ml[(item0 + i0 + i) * H + h].x - M);
+#pragma unroll
+            for (int j = 0; j < DPL; ++j) o[j] = fmaf(wgt, a[i][j], o[j]);
+          }
+        }
       }
       const float invL = 1.f / Lh;
       T* out = reinterpret_cast<T*>(p.out) + (((long long)l_rel * B + b) * H + h) * D;
@@ -583,8 +612,7 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
     }
   }
   __syncthreads();
-  const long long lb = (long long)l * B + b;
-  const int n_cur = p.n_cur[lb];
+  const int n_cur = n_dev;
   if (n_cur != p.ncur[l_rel]) {  // host bookkeeping and device state disagree: flag, do not touch
     if (tid == 0) atomicOr(p.status, ST3_DEV_COUNT_MISMATCH);
     return;
@@ -599,18 +627,40 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   float* mass_by_id = p.mass_by_id + lb * Nv;
 
   // ---- visual scores: probability of every visual row summed over heads ----
-  bool bad = false;
-  for (int i = tid; i < n_cur; i += kFinishThreads) {
-    float mass = 0.f;
-    const float* lg = p.logits + lb * H * Nv + i;
-    for (int h = 0; h < H; ++h) mass += fast_exp2(lg[(long long)h * Nv] - s_M[h]) * s_invL[h];
-    if (!(mass >= 0.f) || !(mass <= 3.0e38f)) { bad = true; mass = 0.f; }
-    const int id = ids[i];
-    mass_by_id[id] = mass;
-    s_key[i] = ((unsigned long long)__float_as_uint(mass) << 32) | (unsigned long long)(0xffffffffu - (unsigned)id);
+  // Thread (row r, half g) sums 16 heads at a time with all 16 loads in flight; half 1 hands its
+  // sum to half 0 through shared memory, so the order of the additions is fixed.
+  {
+    constexpr int kRowsPerPass = kFinishThreads / 2, kHeadBatch = 16;
+    const int ri = tid % kRowsPerPass, hg = tid / kRowsPerPass;
+    bool bad = false;
+    for (int i0 = 0; i0 < n_cur; i0 += kRowsPerPass) {
+      const int i = i0 + ri;
+      float pm = 0.f;
+      int id = 0;
+      if (i < n_cur) {
+        if (hg == 0) id = ids[i];
+        const float* lg = p.logits + lb * H * Nv + i;
+        for (int h0 = hg * kHeadBatch; h0 < H; h0 += 2 * kHeadBatch) {
+          float v[kHeadBatch];
+#pragma unroll
+          for (int j = 0; j < kHeadBatch; ++j) v[j] = h0 + j < H ? lg[(long long)(h0 + j) * Nv] : -INFINITY;
+#pragma unroll
+          for (int j = 0; j < kHeadBatch; ++j)
+            if (h0 + j < H) pm += fast_exp2(v[j] - s_M[h0 + j]) * s_invL[h0 + j];
+        }
+      }
+      if (hg == 1) s_half[ri] = pm;
+      __syncthreads();
+      if (hg == 0 && i < n_cur) {
+        float mass = pm + s_half[ri];
+        if (!(mass >= 0.f) || !(mass <= 3.0e38f)) { bad = true; mass = 0.f; }
+        mass_by_id[id] = mass;
+        s_key[i] = ((unsigned long long)__float_as_uint(mass) << 32) | (unsigned long long)(0xffffffffu - (unsigned)id);
+      }
+      __syncthreads();
+    }
+    if (bad) atomicOr(p.status, ST3_DEV_NONFINITE);
   }
-  if (bad) atomicOr(p.status, ST3_DEV_NONFINITE);
-  __syncthreads();
 
   // ---- radix select: the k-th largest 64-bit key (keys are unique: ids are) ----
   unsigned long long prefix = 0ull, mask = 0ull;
@@ -694,6 +744,7 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
 
   // ---- move the rows (sources are rows >= k, destinations rows < k: disjoint) ----
   unsigned char* blk0 = reinterpret_cast<unsigned char*>(p.cache) + (size_t)(lb * H) * p.lbh_stride * sizeof(T);
+  const int id_moved = tid < nmove ? ids[s_mover[tid]] : 0;  // in flight together with the rows
   const long long nvec = (long long)nmove * H * 2 * VPR;
   for (long long v = tid; v < nvec; v += kFinishThreads) {
     const int c = (int)(v % VPR);
@@ -705,7 +756,8 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
     const uint4 val = *reinterpret_cast<const uint4*>(base + (size_t)s_mover[j] * ROWB + c * 16);
     *reinterpret_cast<uint4*>(base + (size_t)s_hole[j] * ROWB + c * 16) = val;
   }
-  for (int j = tid; j < nmove; j += kFinishThreads) ids[s_hole[j]] = ids[s_mover[j]];
+  if (tid < nmove) ids[s_hole[tid]] = id_moved;
+  for (int j = tid + kFinishThreads; j < nmove; j += kFinishThreads) ids[s_hole[j]] = ids[s_mover[j]];
   if (tid == 0) p.n_cur[lb] = k;
 }
 

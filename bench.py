@@ -243,12 +243,26 @@ def timed(fn, n, dist):
     torch.cuda.synchronize()
     if dist:
         torch.distributed.barrier()
-    ms = e0.elapsed_time(e1)
-    if dist:
-        t = torch.tensor([ms], device="cuda")
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms = float(t.item())
-    return ms
+    return max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
+
+
+def max_over_ranks(value, dist, device):
+    """The slowest rank's time: what a multi-GPU number is reported on."""
+    if not dist:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_workload(wl, rank, world):
+    """Replicas work on different data: rank r of a multi-GPU run uses seed + 1000 r."""
+    return wl if world == 1 else wl.scaled(seed=wl.seed + 1000 * rank)
+
+
+def job_value(tokens_per_gen, steps, world, ms):
+    """Whole-job tokens/s: every rank processed tokens_per_gen * steps tokens in `ms` (max over ranks)."""
+    return world * tokens_per_gen * steps / (ms * 1e-3)
 
 
 def oracle_sample(wl, g, K, V, q0, q, kn, vn, nsteps, warm_steps, reps=1):
@@ -294,7 +308,7 @@ def main():
     ap.add_argument("--workload", default="llava15_7b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows-per-chunk", type=int, default=0)
-    ap.add_argument("--no-extras", action="store_true", help="skip unpruned / cpu_baseline / e2e legs")
+    ap.add_argument("--no-extras", action="store_true", help="skip the e2e, unpruned and cpu_baseline legs")
     args = ap.parse_args()
     wl = get_workload(args.workload)
     rank = int(os.environ.get("RANK", "0"))
@@ -317,7 +331,6 @@ def main():
         need = n_timed + n_warm
         L = wl.num_layers
         q0 = g.queries([0])[0]
-        K = torch.cat([g.prompt_kv([l])[0] for l in range(L)]) if False else None
         Ks, Vs = zip(*[g.prompt_kv([l]) for l in range(L)])
         K, V = torch.cat(Ks), torch.cat(Vs)
         steps = list(range(1, need + 1))
@@ -343,8 +356,7 @@ def main():
     device = torch.device(f"cuda:{local}")
     if dist:
         torch.distributed.init_process_group("nccl", device_id=device)
-    if dist:
-        wl = wl.scaled(seed=wl.seed + 1000 * rank)       # replicas work on different data
+    wl = replica_workload(wl, rank, world)
     job = Job(wl, device, rows_per_chunk=args.rows_per_chunk)
     B = job.B
     tokens_per_gen = wl.batch * wl.decode_steps
@@ -361,7 +373,7 @@ def main():
     launches = job.ctx.launch_count() - n0
     clocks = sampler.stop() if rank == 0 else None
     job.ctx.status()
-    value = world * tokens_per_gen * args.steps / (ms * 1e-3)
+    value = job_value(tokens_per_gen, args.steps, world, ms)
 
     # per-kernel time of the attention kernel (events around it inside the library), same work
     B.st3_profile_enable(job.ctx.handle, True)
@@ -385,14 +397,15 @@ def main():
             "gpu_launches": int(launches), "roofline": roofline, "clocks": clocks}
 
     # end to end: every input starts in pinned host memory, every output ends there
-    job.make_host()
-    for _ in range(2):
-        job.generation_host()
-    ms_e2e = timed(job.generation_host, args.steps, dist)
-    job.ctx.status()
-    line["e2e"] = {"value": world * tokens_per_gen * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
-                   "h2d_bytes_per_step": job.h2d_bytes(), "d2h_bytes_per_step": job.d2h_bytes(),
-                   "ms_per_step": ms_e2e / args.steps}
+    if not args.no_extras:
+        job.make_host()
+        for _ in range(2):
+            job.generation_host()
+        ms_e2e = timed(job.generation_host, args.steps, dist)
+        job.ctx.status()
+        line["e2e"] = {"value": job_value(tokens_per_gen, args.steps, world, ms_e2e), "unit": UNIT,
+                       "h2d_bytes_per_step": job.h2d_bytes(), "d2h_bytes_per_step": job.d2h_bytes(),
+                       "ms_per_step": ms_e2e / args.steps}
 
     if rank == 0 and world == 1 and not args.no_extras:
         # the same kernels with trimming disabled (full KV cache)

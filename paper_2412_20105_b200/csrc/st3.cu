@@ -65,6 +65,7 @@ struct StepParams {
   int ct;                   // text chunks per (l, b, h), the same for every sequence
   int chunk_rows;           // rows per work item (<= the kernel's tile capacity)
   int total_work;           // work items x heads of this launch
+  int first_dynamic;        // managers of the attention grid: items below this index are pre-assigned
   unsigned h_mul, h_shift;  // fast division by H
   int cvp[kMaxLayers + 1];  // prefix sum of visual chunks per layer (relative layer index)
   int lstart[kMaxLayers + 1];       // first work item of each layer: B * (cvp[l] + l * ct)
@@ -296,8 +297,9 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
       uint4 nv[NV];
     };
     int lcur = 0;  // layer of the previous item: this warp's items arrive in increasing order
-    int x_next = 0;
-    if (lane == 0) x_next = atomicAdd(p.work_counter, 1);
+    // the first item of every manager is fixed (no round trip to the counter before the first copy);
+    // the counter starts behind those and hands out the rest
+    int x_next = (int)blockIdx.x * kSlots + s;
 
     auto decode = [&](Dec& d) {
       const int x = __shfl_sync(0xffffffffu, x_next, 0);
@@ -550,7 +552,7 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   const int B = p.B, H = p.H, Nv = p.Nv;
   const int l_rel = blockIdx.x / B, b = blockIdx.x % B;
   const int l = p.layer_begin + l_rel;
-  if (blockIdx.x == 0 && tid == 0) *p.work_counter = 0;  // the next attention launch starts from item 0
+  if (blockIdx.x == 0 && tid == 0) *p.work_counter = p.first_dynamic;  // ready for the next attention launch
 
   const long long lb = (long long)l * B + b;
   const int n_dev = p.n_cur[lb];  // needed only after the merge: the load overlaps it
@@ -1017,6 +1019,7 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
   const long long total_items = (long long)c.batch * (p.cvp[layer_count] + (long long)layer_count * p.ct);
   if (total_items > L.max_items || total_items * c.num_heads > 0x3fffffffLL) return ST3_ERR_CAPACITY;
   p.total_work = (int)(total_items * c.num_heads);
+  p.first_dynamic = ctx->num_sms * ctx->attend_ctas_per_sm * kSlots;
 
 #define ST3_LAUNCH(T, D) launch_step_t<T, D>(ctx, p, (int)total_items, st, k, v, prefill)
   const st3_status s = ST3_DISPATCH(ctx, ST3_LAUNCH);
@@ -1088,7 +1091,11 @@ st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, 
 #undef ST3_ATTR
   if (s == ST3_OK) {
     // bookkeeping area (scores, ids, counts, text lengths, status word) starts cleared
+    // ... except the work counter, which starts behind the pre-assigned first item of every manager
+    const int first_dynamic = ctx->num_sms * ctx->attend_ctas_per_sm * kSlots;
     if (cudaMemsetAsync(ctx->ws + L.mass, 0, L.stage_q - L.mass, nullptr) != cudaSuccess ||
+        cudaMemcpyAsync(ctx->ws + L.status + 16 * sizeof(int), &first_dynamic, sizeof(int), cudaMemcpyHostToDevice,
+                        nullptr) != cudaSuccess ||
         cudaStreamSynchronize(nullptr) != cudaSuccess)
       s = ST3_ERR_CUDA;
   }

@@ -37,7 +37,6 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kFinishThreads = 1024;
-constexpr int kFinishWarps = kFinishThreads / 32;
 constexpr int kMaxChunkRows = 128;  // upper bound on the rows of one work item
 constexpr int kMaxLayers = 64;
 constexpr int kMaxHeads = 128;
@@ -536,36 +535,62 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
 // ------------------------------------------------------------------------------------------
 // Merge partials, visual scores, top-k (Eq. 3), in-place compaction (Eq. 7's eviction)
 // ------------------------------------------------------------------------------------------
+// Two blocks per (layer, sequence), on different SMs, that never wait for each other:
+//   OUT block   merges the chunk partials of every head into the attention output (a warp per head);
+//   TRIM block  merges only the (max, sum) pairs, turns the raw logits into head-summed
+//               probabilities, radix-selects the rows to keep, pairs holes with kept tail rows and
+//               moves the rows.
+// Both are chains of dependent memory round trips, so every phase issues all its loads first.
+constexpr int kFinishWarps = kFinishThreads / 32;
+constexpr int kHeadBatch = 16;  // logits of one visual row a thread keeps in flight
+
+// (max, 1/sum) of one head's merged softmax from its chunk partials; every lane gets both.
+__device__ __forceinline__ void merge_stats(const float2* ml, long long item0, int nit, int H, int h, int lane,
+                                            float& M, float& L) {
+  float2 v[2];  // the first 64 partials stay in registers
+#pragma unroll
+  for (int j = 0; j < 2; ++j)
+    v[j] = lane + 32 * j < nit ? ml[(item0 + lane + 32 * j) * H + h] : make_float2(-INFINITY, 0.f);
+  M = fmaxf(v[0].x, v[1].x);
+  for (int i = lane + 64; i < nit; i += 32) M = fmaxf(M, ml[(item0 + i) * H + h].x);
+  M = warp_max(M);
+  L = v[0].y * fast_exp2(v[0].x - M) + v[1].y * fast_exp2(v[1].x - M);
+  for (int i = lane + 64; i < nit; i += 32) {
+    const float2 u = ml[(item0 + i) * H + h];
+    L += u.y * fast_exp2(u.x - M);
+  }
+  L = warp_sum(L);
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepParams p) {
   constexpr int ROWB = D * sizeof(T);
   constexpr int VPR = ROWB / 16;  // 16-byte vectors per row
+  constexpr int DPL = D / 32;
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ float s_M[kMaxHeads];
   __shared__ float s_invL[kMaxHeads];
   __shared__ int s_hist[256];
   __shared__ int s_scan[kFinishWarps];
-  __shared__ int s_sel[3];  // digit, count above, count in bin
   __shared__ float s_half[kFinishThreads / 2];
+  __shared__ int s_sel[3];  // digit, count above, count in bin
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x, lane = tid & 31;
   const int B = p.B, H = p.H, Nv = p.Nv;
-  const int l_rel = blockIdx.x / B, b = blockIdx.x % B;
+  const int units = p.layer_count * B;  // blocks [0, units) trim, blocks [units, 2 units) write the output
+  const bool out_role = (int)blockIdx.x >= units;
+  const int unit = out_role ? blockIdx.x - units : blockIdx.x;
+  const int l_rel = unit / B, b = unit % B;
   const int l = p.layer_begin + l_rel;
-  if (blockIdx.x == 0 && tid == 0) *p.work_counter = p.first_dynamic;  // ready for the next attention launch
-
   const long long lb = (long long)l * B + b;
-  const int n_dev = p.n_cur[lb];  // needed only after the merge: the load overlaps it
+  const int nit = p.cvp[l_rel + 1] - p.cvp[l_rel] + p.ct;
+  const long long item0 = (long long)p.lstart[l_rel] + (long long)b * nit;
+  const float2* ml = reinterpret_cast<const float2*>(p.part_ml);
 
-  // ---- merge the chunk partials of every head (one warp per head) ----
-  // Loads are issued in batches so that a head costs one memory round trip per kMergeBatch partials.
-  {
-    constexpr int DPL = D / 32;
-    constexpr int kMergeBatch = 8;
-    const int nit = p.cvp[l_rel + 1] - p.cvp[l_rel] + p.ct;
-    const long long item0 = (long long)p.lstart[l_rel] + (long long)b * nit;
-    const float2* ml = reinterpret_cast<const float2*>(p.part_ml);
-    for (int h = warp; h < H; h += kFinishWarps) {
+  if (out_role) {
+    // ===================== OUT block: attention output of every head =====================
+    constexpr int kMergeBatch = 8;  // partials in flight per round trip
+    for (int h = tid >> 5; h < H; h += kFinishWarps) {
       float a[kMergeBatch][DPL];
       auto load_batch = [&](int i0) {
 #pragma unroll
@@ -583,15 +608,8 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
         }
       };
       load_batch(0);
-      float M = -INFINITY;
-      for (int i = lane; i < nit; i += 32) M = fmaxf(M, ml[(item0 + i) * H + h].x);
-      M = warp_max(M);
-      float Lh = 0.f;
-      for (int i = lane; i < nit; i += 32) {
-        const float2 v = ml[(item0 + i) * H + h];
-        Lh += v.y * fast_exp2(v.x - M);
-      }
-      Lh = warp_sum(Lh);
+      float M, Lh;
+      merge_stats(ml, item0, nit, H, h, lane, M, Lh);
       float o[DPL];
 #pragma unroll
       for (int j = 0; j < DPL; ++j) o[j] = 0.f;
@@ -610,68 +628,97 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
       T* out = reinterpret_cast<T*>(p.out) + (((long long)l_rel * B + b) * H + h) * D;
 #pragma unroll
       for (int j = 0; j < DPL; ++j) store_out(out + lane * DPL + j, o[j] * invL);
-      if (lane == 0) { s_M[h] = M; s_invL[h] = invL; }
     }
-  }
-  __syncthreads();
-  const int n_cur = n_dev;
-  if (n_cur != p.ncur[l_rel]) {  // host bookkeeping and device state disagree: flag, do not touch
-    if (tid == 0) atomicOr(p.status, ST3_DEV_COUNT_MISMATCH);
     return;
   }
-  const int k = min(n_cur, p.ntgt[l_rel]);
-  if (k >= n_cur) return;
 
+  // ===================== TRIM block =====================
+  const int tt = tid, warp = tid >> 5;
+  if (blockIdx.x == 0 && tt == 0) *p.work_counter = p.first_dynamic;  // ready for the next attention launch
+  const int n_host = p.ncur[l_rel];
+  const int k = min(n_host, p.ntgt[l_rel]);
+  const bool evicts = k < n_host;  // same answer in every thread
+  const int n_dev = p.n_cur[lb];
+  if (!evicts) {
+    if (tt == 0 && n_dev != n_host) atomicOr(p.status, ST3_DEV_COUNT_MISMATCH);
+    return;
+  }
+  int* ids = p.ids + lb * Nv;
+  float* mass_by_id = p.mass_by_id + lb * Nv;
+  const float* logits = p.logits + lb * H * Nv;
   unsigned long long* s_key = reinterpret_cast<unsigned long long*>(smem);  // [Nv]
   int* s_hole = reinterpret_cast<int*>(smem + (size_t)Nv * 8);              // [Nv]
   int* s_mover = s_hole + Nv;                                               // [Nv]
-  int* ids = p.ids + lb * Nv;
-  float* mass_by_id = p.mass_by_id + lb * Nv;
+  const int n_cur = n_host;
+
+  // Thread (row r, half g) of a pass sums every second batch of 16 heads of its row; half 1 hands its
+  // sum to half 0 through shared memory, so the order of the additions is fixed.  The first batch of
+  // the first pass is requested now, together with the (max, sum) pairs: one round trip for both.
+  constexpr int kRowsPerPass = kFinishThreads / 2;
+  const int ri = tt % kRowsPerPass, hg = tt / kRowsPerPass;
+  float pre[kHeadBatch];
+  int id0 = 0;
+  if (ri < n_cur) {
+    if (hg == 0) id0 = ids[ri];
+#pragma unroll
+    for (int j = 0; j < kHeadBatch; ++j) {
+      const int h = hg * kHeadBatch + j;
+      pre[j] = h < H ? logits[(long long)h * Nv + ri] : -INFINITY;
+    }
+  }
+  for (int h = warp; h < H; h += kFinishWarps) {
+    float M, Lh;
+    merge_stats(ml, item0, nit, H, h, lane, M, Lh);
+    if (lane == 0) { s_M[h] = M; s_invL[h] = 1.f / Lh; }
+  }
+  __syncthreads();
+  if (n_dev != n_host) {  // host bookkeeping and device state disagree: flag, do not touch
+    if (tt == 0) atomicOr(p.status, ST3_DEV_COUNT_MISMATCH);
+    return;
+  }
 
   // ---- visual scores: probability of every visual row summed over heads ----
-  // Thread (row r, half g) sums 16 heads at a time with all 16 loads in flight; half 1 hands its
-  // sum to half 0 through shared memory, so the order of the additions is fixed.
-  {
-    constexpr int kRowsPerPass = kFinishThreads / 2, kHeadBatch = 16;
-    const int ri = tid % kRowsPerPass, hg = tid / kRowsPerPass;
-    bool bad = false;
-    for (int i0 = 0; i0 < n_cur; i0 += kRowsPerPass) {
-      const int i = i0 + ri;
-      float pm = 0.f;
-      int id = 0;
-      if (i < n_cur) {
-        if (hg == 0) id = ids[i];
-        const float* lg = p.logits + lb * H * Nv + i;
-        for (int h0 = hg * kHeadBatch; h0 < H; h0 += 2 * kHeadBatch) {
-          float v[kHeadBatch];
+  bool bad = false;
+  for (int i0 = 0; i0 < n_cur; i0 += kRowsPerPass) {
+    const int i = i0 + ri;
+    float pm = 0.f;
+    int id = id0;
+    if (i < n_cur) {
+      if (i0 && hg == 0) id = ids[i];
+      for (int h0 = hg * kHeadBatch; h0 < H; h0 += 2 * kHeadBatch) {
+        float v[kHeadBatch];
+        if (i0 == 0 && h0 == hg * kHeadBatch) {
 #pragma unroll
-          for (int j = 0; j < kHeadBatch; ++j) v[j] = h0 + j < H ? lg[(long long)(h0 + j) * Nv] : -INFINITY;
+          for (int j = 0; j < kHeadBatch; ++j) v[j] = pre[j];
+        } else {
 #pragma unroll
-          for (int j = 0; j < kHeadBatch; ++j)
-            if (h0 + j < H) pm += fast_exp2(v[j] - s_M[h0 + j]) * s_invL[h0 + j];
+          for (int j = 0; j < kHeadBatch; ++j) v[j] = h0 + j < H ? logits[(long long)(h0 + j) * Nv + i] : -INFINITY;
         }
+#pragma unroll
+        for (int j = 0; j < kHeadBatch; ++j)
+          if (h0 + j < H) pm += fast_exp2(v[j] - s_M[h0 + j]) * s_invL[h0 + j];
       }
-      if (hg == 1) s_half[ri] = pm;
-      __syncthreads();
-      if (hg == 0 && i < n_cur) {
-        float mass = pm + s_half[ri];
-        if (!(mass >= 0.f) || !(mass <= 3.0e38f)) { bad = true; mass = 0.f; }
-        mass_by_id[id] = mass;
-        s_key[i] = ((unsigned long long)__float_as_uint(mass) << 32) | (unsigned long long)(0xffffffffu - (unsigned)id);
-      }
-      __syncthreads();
     }
-    if (bad) atomicOr(p.status, ST3_DEV_NONFINITE);
+    if (hg == 1) s_half[ri] = pm;
+    __syncthreads();
+    if (hg == 0 && i < n_cur) {
+      float mass = pm + s_half[ri];
+      if (!(mass >= 0.f) || !(mass <= 3.0e38f)) { bad = true; mass = 0.f; }
+      mass_by_id[id] = mass;
+      s_key[i] = ((unsigned long long)__float_as_uint(mass) << 32) | (unsigned long long)(0xffffffffu - (unsigned)id);
+    }
+    __syncthreads();
   }
+  if (bad) atomicOr(p.status, ST3_DEV_NONFINITE);
 
   // ---- radix select: the k-th largest 64-bit key (keys are unique: ids are) ----
   unsigned long long prefix = 0ull, mask = 0ull;
   if (k > 0) {
     int need = k;
     for (int shift = 56; shift >= 0; shift -= 8) {
-      if (tid < 256) s_hist[tid] = 0;
+      if (tt < 256) s_hist[tt] = 0;
       __syncthreads();
-      for (int i = tid; i < n_cur; i += kFinishThreads) {
+      for (int i = tt; i < n_cur; i += kFinishThreads) {
         const unsigned long long key = s_key[i];
         if ((key & mask) == prefix) atomicAdd(&s_hist[(int)((key >> shift) & 0xffull)], 1);
       }
@@ -708,7 +755,7 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
 
   // ---- pair every hole among the first k rows with a kept row of the tail ----
   const int per = (n_cur + kFinishThreads - 1) / kFinishThreads;
-  const int i0 = min(n_cur, tid * per), i1 = min(n_cur, i0 + per);
+  const int i0 = min(n_cur, tt * per), i1 = min(n_cur, i0 + per);
   int nh = 0, nm = 0;
   for (int i = i0; i < i1; ++i) {
     const bool keep = s_key[i] >= prefix;
@@ -740,15 +787,15 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   __syncthreads();
   const int nmove = total & 0xffff;
   if (nmove != (total >> 16)) {  // cannot happen when exactly k keys pass the threshold
-    if (tid == 0) atomicOr(p.status, ST3_DEV_RANGE);
+    if (tt == 0) atomicOr(p.status, ST3_DEV_RANGE);
     return;
   }
 
   // ---- move the rows (sources are rows >= k, destinations rows < k: disjoint) ----
+  const int id_moved = tt < nmove ? ids[s_mover[tt]] : 0;  // in flight together with the rows
   unsigned char* blk0 = reinterpret_cast<unsigned char*>(p.cache) + (size_t)(lb * H) * p.lbh_stride * sizeof(T);
-  const int id_moved = tid < nmove ? ids[s_mover[tid]] : 0;  // in flight together with the rows
   const long long nvec = (long long)nmove * H * 2 * VPR;
-  for (long long v = tid; v < nvec; v += kFinishThreads) {
+  for (long long v = tt; v < nvec; v += kFinishThreads) {
     const int c = (int)(v % VPR);
     long long r = v / VPR;
     const int kv = (int)(r % 2); r /= 2;
@@ -758,9 +805,9 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
     const uint4 val = *reinterpret_cast<const uint4*>(base + (size_t)s_mover[j] * ROWB + c * 16);
     *reinterpret_cast<uint4*>(base + (size_t)s_hole[j] * ROWB + c * 16) = val;
   }
-  if (tid < nmove) ids[s_hole[tid]] = id_moved;
-  for (int j = tid + kFinishThreads; j < nmove; j += kFinishThreads) ids[s_hole[j]] = ids[s_mover[j]];
-  if (tid == 0) p.n_cur[lb] = k;
+  if (tt < nmove) ids[s_hole[tt]] = id_moved;
+  for (int j = tt + kFinishThreads; j < nmove; j += kFinishThreads) ids[s_hole[j]] = ids[s_mover[j]];
+  if (tt == 0) p.n_cur[lb] = k;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -953,7 +1000,7 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
   (void)total_items;
   st3_attend_kernel<T, D><<<(unsigned)(ctx->num_sms * ctx->attend_ctas_per_sm), kAttendThreads, ctx->attend_smem, st>>>(p);
   if (e1) cudaEventRecord(e1, st);
-  st3_finish_kernel<T, D><<<(unsigned)(p.layer_count * c.batch), kFinishThreads, ctx->finish_smem, st>>>(p);
+  st3_finish_kernel<T, D><<<(unsigned)(2 * p.layer_count * c.batch), kFinishThreads, ctx->finish_smem, st>>>(p);
   if (e2) cudaEventRecord(e2, st);
   ctx->launches += 2;
   return cudaGetLastError() == cudaSuccess ? ST3_OK : ST3_ERR_CUDA;

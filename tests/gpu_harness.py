@@ -31,10 +31,10 @@ def assert_out_close(got: np.ndarray, ref: np.ndarray, dtype: str, where=""):
 
 
 class GpuRun:
-    def __init__(self, wl: Workload, device="cuda:0", **cfg_overrides):
+    def __init__(self, wl: Workload, device="cuda:0", sched_kw=None, **cfg_overrides):
         self.wl, self.dev = wl, torch.device(device)
         self.g = SynthInputs(wl)
-        self.sched = make_schedule(wl, disable_trim=bool(cfg_overrides.get("disable_trim", 0)))
+        self.sched = make_schedule(wl, disable_trim=bool(cfg_overrides.get("disable_trim", 0)), **(sched_kw or {}))
         self.cfg = B.config_from_workload(wl, **cfg_overrides)
         self.ctx = B.Context(self.cfg, device)
         self.L = wl.num_layers

@@ -1,0 +1,158 @@
+"""Behaviour of the C ABI on a GPU beyond plain parity: host-buffer step, call-order errors,
+context reuse, bookkeeping queries, profiling counters, schedule variants."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2412_20105_b200 import binding as B
+from synth import SynthInputs, get_workload
+from gpu_harness import GpuRun, run_and_check
+from helpers import make_schedule
+
+pytestmark = pytest.mark.gpu
+
+
+def _small(**kw):
+    base = dict(dtype="bf16", head_dim=128, num_heads=4, num_layers=6, batch=2, sys_len=5, num_visual=200,
+                text_len_min=3, text_len_max=20, decode_steps=12, first_prune_layer=2, stride=2,
+                step_ratio_bp=1500, tau=12.0, num_planted=10)
+    base.update(kw)
+    return get_workload("tiny").scaled(**base)
+
+
+def test_host_buffer_step_equals_device_step():
+    wl = _small()
+    a, b = GpuRun(wl), GpuRun(wl)
+    try:
+        a.prefill(); b.prefill()
+        assert torch.equal(a.out, b.out)
+        for t in range(1, 6):
+            a.decode(t)
+            q, kn, vn = b.inputs(t)
+            hq, hk, hv = (x.cpu().pin_memory() for x in (q, kn, vn))
+            hout = torch.empty_like(hq).pin_memory()
+            b.ctx.decode_step_host(t, hq, hk, hv, hout)
+            torch.cuda.synchronize()
+            assert torch.equal(hout, a.out.cpu()), t
+            for l in range(wl.num_layers):
+                ia, ca, _ = a.kept(l)
+                ib, cb, _ = b.kept(l)
+                assert np.array_equal(ca, cb)
+                for s in range(wl.batch):
+                    assert np.array_equal(ia[s, :ca[s]], ib[s, :cb[s]])
+        assert a.ctx.status() == 0 and b.ctx.status() == 0
+    finally:
+        a.close(); b.close()
+
+
+def test_call_order_and_capacity_errors():
+    wl = _small()
+    run = GpuRun(wl)
+    try:
+        q, kn, vn = run.inputs(1)
+        with pytest.raises(B.St3Error) as e:                      # decode before any prefill
+            run.ctx.decode_step(1, q, kn, vn, run.out)
+        assert e.value.code == 3
+        run.prefill()
+        with pytest.raises(B.St3Error) as e:                      # step gap
+            run.ctx.decode_step(2, q, kn, vn, run.out)
+        assert e.value.code == 3
+        run.ctx.decode_step(1, q, kn, vn, run.out)
+        with pytest.raises(B.St3Error) as e:                      # same step twice
+            run.ctx.decode_step(1, q, kn, vn, run.out)
+        assert e.value.code == 3
+        with pytest.raises(B.St3Error) as e:                      # beyond max_decode_steps
+            run.ctx.decode_step(wl.decode_steps + 1, q, kn, vn, run.out)
+        assert e.value.code == 4
+        with pytest.raises(B.St3Error) as e:                      # layer range out of bounds
+            run.ctx.decode_step(2, q, kn, vn, run.out, layer_begin=1)
+        assert e.value.code == 1
+        with pytest.raises(B.St3Error) as e:                      # text longer than the configured maximum
+            B.st3_prefill_select(run.ctx.handle, 0, wl.num_layers, run.q_cur.data_ptr(), run.q_cur.data_ptr(),
+                                 run.q_cur.data_ptr(), [wl.text_len_max + 1] * wl.batch, run.out.data_ptr(), 0)
+        assert e.value.code == 4
+        with pytest.raises(B.St3Error) as e:                      # misaligned pointer
+            B.st3_decode_step(run.ctx.handle, 2, 0, wl.num_layers, q.data_ptr() + 2, kn.data_ptr(), vn.data_ptr(),
+                              run.out.data_ptr(), 0)
+        assert e.value.code == 1
+        # the failed calls changed nothing: step 2 still works and still matches the oracle
+        before = run.snapshot(range(wl.num_layers))
+        run.decode(2)
+        for l in range(wl.num_layers):
+            run.check_decode_unit(0, l, 2, before[l])
+        assert run.ctx.status() == 0
+    finally:
+        run.close()
+
+
+def test_context_is_reusable_for_a_new_generation():
+    wl = _small()
+    run = GpuRun(wl)
+    try:
+        run.prefill()
+        for t in range(1, 5):
+            run.decode(t)
+        first = {l: run.kept(l) for l in range(wl.num_layers)}
+        out_first = run.out.clone()
+        run.prefill()                                             # same prompt again: state starts over
+        for t in range(1, 5):
+            run.decode(t)
+        assert torch.equal(out_first, run.out)
+        for l in range(wl.num_layers):
+            ids, cnt, _ = run.kept(l)
+            assert np.array_equal(cnt, first[l][1])
+            for s in range(wl.batch):
+                assert np.array_equal(ids[s, :cnt[s]], first[l][0][s, :cnt[s]])
+        assert run.ctx.status() == 0
+    finally:
+        run.close()
+
+
+def test_rows_held_and_launch_counters_follow_the_schedule():
+    wl = _small()
+    run = GpuRun(wl)
+    try:
+        assert run.ctx.rows_held() == (0, 0)
+        n0 = run.ctx.launch_count()
+        run.prefill()
+        assert run.ctx.launch_count() - n0 == 3                   # ingest, attend, finish
+        sched = make_schedule(wl)
+        text = run.g.text_len
+        for t in range(0, 4):
+            if t:
+                run.decode(t)
+            vis, oth = run.ctx.rows_held()
+            assert vis == wl.batch * sum(sched.n(l, t) for l in range(wl.num_layers))
+            assert oth == wl.num_layers * sum(wl.sys_len + int(x) + t for x in text)
+        assert run.ctx.launch_count() - n0 == 3 + 2 * 3
+        B.st3_profile_enable(run.ctx.handle, True)
+        run.decode(4); run.decode(5)
+        a_ms, f_ms, na, nf = B.st3_profile_read(run.ctx.handle)
+        assert na == nf == 2 and a_ms > 0 and f_ms > 0
+        B.st3_profile_enable(run.ctx.handle, False)
+        assert run.ctx.status() == 0
+    finally:
+        run.close()
+
+
+@pytest.mark.parametrize("anneal,kw", [("linear", dict(tau=12.0)), ("exp", dict(sigma=4.0)), ("none", dict())])
+def test_other_attenuation_functions(anneal, kw):
+    code = {"linear": B.ST3_ANNEAL_LINEAR, "exp": B.ST3_ANNEAL_EXP, "none": B.ST3_ANNEAL_NONE}[anneal]
+    wl = _small(**{k: v for k, v in kw.items() if k == "tau"})
+    stats = run_and_check(wl, wl.decode_steps, sched_kw=dict(anneal=anneal, **{k: v for k, v in kw.items() if k == "sigma"}),
+                          anneal=code, **{k: v for k, v in kw.items() if k == "sigma"})
+    assert stats["units"] == (wl.decode_steps + 1) * wl.num_layers * wl.batch
+
+
+def test_layer_by_layer_calls_match_one_call_for_all_layers():
+    wl = _small()
+    a, b = GpuRun(wl), GpuRun(wl)
+    try:
+        a.prefill(); b.prefill(layers_per_call=1)
+        assert torch.equal(a.out, b.out)
+        for t in range(1, 5):
+            a.decode(t); b.decode(t, layers_per_call=1)
+            assert torch.equal(a.out, b.out), t
+        assert a.ctx.status() == 0 and b.ctx.status() == 0
+    finally:
+        a.close(); b.close()

@@ -177,12 +177,20 @@ class LayerCache:
         self.ids = self.ids[pos]
 
 
-def prefill_select(q_last, K, V, sys_len: int, num_visual: int, n_keep: int):
+def rank_order(scores: np.ndarray, ids: np.ndarray) -> np.ndarray:
+    """Positions sorted by descending score, equal scores by lower original index: the saved
+    top-index list T[l] of Algorithm 3.  Every prefix of it is a Top(G, .) of Eq. 3."""
+    return np.lexsort((np.asarray(ids), -np.asarray(scores, dtype=np.float64)))
+
+
+def prefill_select(q_last, K, V, sys_len: int, num_visual: int, n_keep: int, rank_ordered: bool = False):
     """Prefill half of Algorithm 3 for one (sequence, layer).
 
     K, V [H, T0, D] hold the prompt rows [S | V | I]; q_last [H, D] is the last
     prompt token's query.  Attends over the whole prompt, scores the visual
     tokens, keeps the n_keep best (Eq. 3) and builds the cache.
+    With rank_ordered the kept rows are stored in the order of the top-index list (best first),
+    which is what the static-rank decode of Algorithm 3 truncates.
     Returns (out [H, D], mass [num_visual], cache).
     """
     K = np.asarray(K, dtype=np.float64)
@@ -190,7 +198,10 @@ def prefill_select(q_last, K, V, sys_len: int, num_visual: int, n_keep: int):
     out, p = attend(q_last, K, V)
     mass = visual_mass(p, sys_len, num_visual)
     ids_all = np.arange(num_visual, dtype=np.int64)
-    kept = select_top(mass, ids_all, n_keep)
+    if rank_ordered:
+        kept = rank_order(mass, ids_all)[:max(0, min(int(n_keep), num_visual))]
+    else:
+        kept = select_top(mass, ids_all, n_keep)
     v0, v1 = sys_len, sys_len + num_visual
     cache = LayerCache(
         K_sys=K[:, :v0].copy(), V_sys=V[:, :v0].copy(),
@@ -228,6 +239,26 @@ def decode_step(cache: LayerCache, q, k_new, v_new, n_target: int):
         cache.ids = cache.ids[kept]
     cache.last_mass = mass
     return out, mass, ids_before
+
+
+def decode_step_static(cache: LayerCache, q, k_new, v_new, n_target: int):
+    """Decode half of Algorithm 3 as printed, for a cache kept in top-index order.
+
+    T' = T[l][: n] and C = C[T'] come first (the visual rows are cut to the first n_target of the
+    saved order, no re-scoring), then the layer attends over what is left plus the new token.
+    Returns out [H, D].
+    """
+    n_new = min(cache.n_cur, int(n_target))
+    cache.K_vis = cache.K_vis[:, :n_new]
+    cache.V_vis = cache.V_vis[:, :n_new]
+    cache.ids = cache.ids[:n_new]
+    k_new = np.asarray(k_new, dtype=np.float64)
+    v_new = np.asarray(v_new, dtype=np.float64)
+    cache.K_txt = np.concatenate([cache.K_txt, k_new[:, None, :]], axis=1)
+    cache.V_txt = np.concatenate([cache.V_txt, v_new[:, None, :]], axis=1)
+    K, V = cache.rows()
+    out, _ = attend(q, K, V)
+    return out
 
 
 def boundary_scores(mass: np.ndarray, ids: np.ndarray, k: int):

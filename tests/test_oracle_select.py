@@ -74,3 +74,38 @@ def test_prefill_and_decode_bookkeeping():
     assert c.n_cur == 0
     o, m, _ = decode_step(c, r.standard_normal((H, D)), kn, vn, 0)
     assert m.shape == (0,) and np.all(np.isfinite(o))
+
+
+def test_rank_order_prefixes_are_the_top_sets():
+    from oracle.st3_oracle import rank_order
+    r = np.random.default_rng(21)
+    scores = r.integers(0, 6, size=30).astype(np.float64)         # ties
+    ids = r.permutation(64)[:30]
+    order = rank_order(scores, ids)
+    assert sorted(order.tolist()) == list(range(30))
+    for a, b in zip(order[:-1], order[1:]):                       # sorted by (score desc, id asc)
+        assert scores[a] > scores[b] or (scores[a] == scores[b] and ids[a] < ids[b])
+    for k in range(31):
+        assert set(order[:k].tolist()) == set(_exhaustive(scores, ids, k).tolist())
+
+
+def test_static_rank_decode_truncates_the_saved_order():
+    from oracle.st3_oracle import decode_step_static, attend
+    r = np.random.default_rng(22)
+    H, D, sys_len, nv, text = 2, 4, 2, 12, 3
+    T0 = sys_len + nv + text
+    K, V = r.standard_normal((H, T0, D)), r.standard_normal((H, T0, D))
+    out, mass, c = prefill_select(r.standard_normal((H, D)), K, V, sys_len, nv, 8, rank_ordered=True)
+    assert np.all(np.diff(mass[c.ids]) <= 0)                      # best first
+    assert np.array_equal(c.K_vis, K[:, sys_len + c.ids])
+    ids0 = c.ids.copy()
+    q, kn, vn = r.standard_normal((H, D)), r.standard_normal((H, D)), r.standard_normal((H, D))
+    o = decode_step_static(c, q, kn, vn, 5)
+    assert np.array_equal(c.ids, ids0[:5])                        # a prefix, nothing re-scored
+    # it attended over exactly [S | first 5 of the order | I | new token]
+    rows = list(range(sys_len)) + (sys_len + ids0[:5]).tolist() + list(range(sys_len + nv, T0))
+    Kx = np.concatenate([K[:, rows], kn[:, None]], axis=1)
+    Vx = np.concatenate([V[:, rows], vn[:, None]], axis=1)
+    assert np.allclose(o, attend(q, Kx, Vx)[0], rtol=1e-13, atol=1e-15)
+    decode_step_static(c, q, kn, vn, 9)                           # never grows
+    assert c.n_cur == 5

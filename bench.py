@@ -151,14 +151,15 @@ def attend_bytes(wl, cfg, B_mod, text_len, step):
 class Job:
     """All device-resident inputs of one workload plus a library context."""
 
-    def __init__(self, wl, device, disable_trim=False, rows_per_chunk=0):
+    def __init__(self, wl, device, disable_trim=False, rows_per_chunk=0, static_rank=False):
         from paper_2412_20105_b200 import binding as B
         from paper_2412_20105_b200.build import build
         build()
         self.B = B
         self.wl, self.dev = wl, device
         self.g = SynthInputs(wl)
-        self.cfg = B.config_from_workload(wl, disable_trim=int(disable_trim), rows_per_chunk=rows_per_chunk)
+        self.cfg = B.config_from_workload(wl, disable_trim=int(disable_trim), rows_per_chunk=rows_per_chunk,
+                                           static_rank=int(static_rank))
         self.ctx = B.Context(self.cfg, device)
         self.lib = B.load()
         L, T = wl.num_layers, wl.decode_steps
@@ -418,6 +419,15 @@ def main():
         line["unpruned"] = {"value": v_full, "unit": UNIT, "speedup_from_trimming": value / v_full}
         full.ctx.close()
         del full
+        # Algorithm 3 as printed: kept rows in top-index order, decode cuts a prefix (no re-scoring)
+        stat = Job(wl, device, static_rank=True, rows_per_chunk=args.rows_per_chunk)
+        for _ in range(3):
+            stat.generation()
+        ms_stat = timed(stat.generation, args.steps, False)
+        stat.ctx.status()
+        line["static_rank"] = {"value": tokens_per_gen * args.steps / (ms_stat * 1e-3), "unit": UNIT}
+        stat.ctx.close()
+        del stat
         # the oracle on the host cores, bounded sample
         ns = 24 if wl.batch == 1 else max(1, 24 // wl.batch)
         K, V, q0 = job.K.cpu(), job.V.cpu(), job.q0.cpu()

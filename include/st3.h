@@ -80,10 +80,18 @@ typedef struct {
   int32_t step_ratio_bp;     /* R in basis points of |V| removed at each later pruning layer    */
   int32_t anneal;            /* st3_anneal                                                      */
   int32_t disable_trim;      /* 1: same kernels, nothing is ever evicted (full-KV comparison)   */
-  int32_t rows_per_chunk;    /* cache rows one thread block attends over (<= 256); 0 = choose   */
+  int32_t rows_per_chunk;    /* cache rows of one work item of the attention kernel; 0 = choose  */
+  int32_t static_rank;       /* 1: Algorithm 3 as printed, see below; 0: re-rank at every step   */
   double tau;                /* Eq. 8: beta = cos(t*pi/(2 tau)) for t < tau, else 0             */
   double sigma;              /* only ST3_ANNEAL_EXP: beta = exp(-t/sigma)                       */
 } st3_config;
+
+/* static_rank = 1 selects the decode half of Algorithm 3 literally: prefill stores the kept visual
+ * rows in the order of the saved top-index list T[l] (best score first, ties toward the lower
+ * original index), and decode step t first cuts the visual rows to the first n(l, t) of that order
+ * (T' = T[l][:n], C = C[T']: no scoring, no selection, no row moves) and then attends.  With
+ * static_rank = 0 (default) every step attends first and then re-ranks the held rows by the current
+ * query's scores. */
 
 /* Scheduled visual-row count n(l, t) of layer `layer` after decode step `step` (0 = after
  * prefill).  Pure host function.  PVTP: layers below first_prune_layer keep everything; layer l

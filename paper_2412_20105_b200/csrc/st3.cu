@@ -73,6 +73,11 @@ struct StepParams {
   unsigned per_shift[kMaxLayers];
   int ncur[kMaxLayers];     // visual rows held before this step (host's schedule bookkeeping)
   int ntgt[kMaxLayers];     // visual rows to hold after this step
+  int nold[kMaxLayers];     // visual rows the device should report before this step
+  const void* k_in;         // prefill only: the caller's prompt tensors [layer_count][B][H][t0_max][D]
+  const void* v_in;
+  int t0_max;
+  int static_rank;          // 1: keep the kept rows in top-index order, cut them without scoring
 };
 
 // ------------------------------------------------------------------------------------------
@@ -640,7 +645,10 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   const bool evicts = k < n_host;  // same answer in every thread
   const int n_dev = p.n_cur[lb];
   if (!evicts) {
-    if (tt == 0 && n_dev != n_host) atomicOr(p.status, ST3_DEV_COUNT_MISMATCH);
+    if (tt == 0) {
+      if (n_dev != p.nold[l_rel]) atomicOr(p.status, ST3_DEV_COUNT_MISMATCH);
+      else if (n_host != n_dev) p.n_cur[lb] = n_host;  // static-rank cut: only the count changes
+    }
     return;
   }
   int* ids = p.ids + lb * Nv;
@@ -751,6 +759,38 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
     }
   } else {
     prefix = ~0ull;  // keep nothing (ids are < 2^31, so no key reaches this value)
+  }
+
+  if (p.static_rank) {
+    // ---- top-index order: the kept row with r larger keys goes to position r, copied from the
+    // caller's prompt tensors (the cache rows are only written, so nothing is read after being moved)
+    for (int i = tt; i < n_cur; i += kFinishThreads) s_mover[i] = ids[i];
+    for (int i = tt; i < n_cur; i += kFinishThreads) {
+      const unsigned long long key = s_key[i];
+      if (key >= prefix) {
+        int r = 0;
+        for (int j = 0; j < n_cur; ++j) r += s_key[j] > key;
+        s_hole[r] = i;
+      }
+    }
+    __syncthreads();
+    unsigned char* blk0 = reinterpret_cast<unsigned char*>(p.cache) + (size_t)(lb * H) * p.lbh_stride * sizeof(T);
+    const long long nvec = (long long)k * H * 2 * VPR;
+    for (long long v = tt; v < nvec; v += kFinishThreads) {
+      const int c = (int)(v % VPR);
+      long long r = v / VPR;
+      const int kv = (int)(r % 2); r /= 2;
+      const int h = (int)(r % H);
+      const int j = (int)(r / H);
+      const unsigned char* src = reinterpret_cast<const unsigned char*>(kv ? p.v_in : p.k_in) +
+                                 ((((size_t)l_rel * B + b) * H + h) * p.t0_max + p.sys_len + s_mover[s_hole[j]]) * ROWB;
+      unsigned char* dst = blk0 + (size_t)h * p.lbh_stride * sizeof(T) + (size_t)kv * Nv * ROWB + (size_t)j * ROWB;
+      *reinterpret_cast<uint4*>(dst + c * 16) = *reinterpret_cast<const uint4*>(src + c * 16);
+    }
+    __syncthreads();  // every thread has read the old ids it needs
+    for (int j = tt; j < k; j += kFinishThreads) ids[j] = s_mover[s_hole[j]];
+    if (tt == 0) p.n_cur[lb] = k;
+    return;
   }
 
   // ---- pair every hole among the first k rows with a kept row of the tail ----
@@ -1046,13 +1086,18 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
   p.layer_begin = layer_begin; p.layer_count = layer_count; p.B = c.batch; p.H = c.num_heads;
   p.sys_len = c.sys_len; p.Nv = c.num_visual; p.cap_txt = L.cap_txt; p.step = step; p.append = prefill ? 0 : 1;
   p.chunk_rows = L.chunk_rows;
+  p.static_rank = c.static_rank ? 1 : 0;
+  p.k_in = prefill ? k : nullptr; p.v_in = prefill ? v : nullptr;
+  p.t0_max = c.sys_len + c.num_visual + c.max_text_len;
   const int R = L.chunk_rows;
   p.ct = ceil_div(c.sys_len + ctx->max_text + step, R);
   p.cvp[0] = 0;
   for (int i = 0; i < layer_count; ++i) {
     const int l = layer_begin + i;
-    const int ncur = prefill ? c.num_visual : ctx->n_host[l];
+    int ncur = prefill ? c.num_visual : ctx->n_host[l];
     const int tgt = ctx->n_tab[(size_t)l * (c.max_decode_steps + 1) + step];
+    p.nold[i] = ncur;
+    if (c.static_rank && !prefill && tgt < ncur) ncur = tgt;  // cut first, then attend (Algorithm 3)
     p.ncur[i] = ncur;
     p.ntgt[i] = tgt < ncur ? tgt : ncur;
     const int cv = ceil_div(ncur, R);

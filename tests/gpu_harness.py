@@ -30,6 +30,18 @@ def assert_out_close(got: np.ndarray, ref: np.ndarray, dtype: str, where=""):
         assert rel.max() <= OUT_REL_BF16, f"{where}: max-rel {rel.max()}"
 
 
+def assert_rank_ordered(ref_mass, got_ids, where="", rel=1e-3):
+    """The stored order is best-first by the oracle's scores; neighbours may swap only inside a near-tie."""
+    m = np.asarray(ref_mass)[np.asarray(got_ids, dtype=np.int64)]
+    for r in range(len(m) - 1):
+        if m[r] > m[r + 1]:
+            continue
+        if m[r] == m[r + 1]:
+            assert got_ids[r] < got_ids[r + 1], f"{where}: equal scores must be ordered by lower index (rank {r})"
+        else:
+            assert m[r + 1] - m[r] <= rel * abs(m[r + 1]), f"{where}: rank {r} out of order: {m[r]} < {m[r + 1]}"
+
+
 class GpuRun:
     def __init__(self, wl: Workload, device="cuda:0", sched_kw=None, **cfg_overrides):
         self.wl, self.dev = wl, torch.device(device)
@@ -40,6 +52,7 @@ class GpuRun:
         self.L = wl.num_layers
         self.out = torch.empty(self.ctx.io_shape(), dtype=self.ctx.dtype, device=self.dev)
         self.stats = {"exact": 0, "near-tie": 0, "units": 0}
+        self.static = bool(cfg_overrides.get("static_rank", 0))
 
     def close(self):
         self.ctx.close()
@@ -97,6 +110,8 @@ class GpuRun:
         assert n == s.n0(l), (n, s.n0(l))
         self._judge(ref_mass, np.arange(wl.num_visual), s.n0(l), ids[b, :n], mass[b], trimmed=s.n0(l) < wl.num_visual,
                     where=f"prefill b={b} l={l}")
+        if self.static and s.n0(l) < wl.num_visual:
+            assert_rank_ordered(ref_mass, ids[b, :n], f"prefill order b={b} l={l}")
 
     def check_decode_unit(self, b, l, step, before):
         """`before` = (ids [B, Nv], count [B]) of layer l taken before the step ran."""
@@ -104,6 +119,17 @@ class GpuRun:
         ids_b, cnt_b = before
         nb = int(cnt_b[b])
         cache = rebuild_cache(wl, g, b, l, ids_b[b, :nb], step - 1)
+        if self.static:
+            ref_out = O.decode_step_static(cache, f64(self.q_cur[l, b]), f64(self.kn_cur[l, b]), f64(self.vn_cur[l, b]),
+                                           s.n(l, step))
+            assert_out_close(f64(self.out[l, b]), ref_out, wl.dtype, f"static decode out b={b} l={l} t={step}")
+            ids, cnt, _ = self.kept(l)
+            n = int(cnt[b])
+            assert n == min(nb, s.n(l, step))
+            assert np.array_equal(ids[b, :n], ids_b[b, :n]), "static-rank cut must keep a prefix of the saved order"
+            self.stats["exact"] += 1
+            self.stats["units"] += 1
+            return
         ref_out, ref_mass, ids_before = O.decode_step(cache, f64(self.q_cur[l, b]), f64(self.kn_cur[l, b]),
                                                       f64(self.vn_cur[l, b]), s.n(l, step))
         assert_out_close(f64(self.out[l, b]), ref_out, wl.dtype, f"decode out b={b} l={l} t={step}")

@@ -80,3 +80,21 @@ def test_full_size_workloads_sampled_units(name, steps):
     lpc = 8 if wl.batch > 1 else None
     stats = run_and_check(wl, wl.decode_steps, check_steps=steps, units=units, layers_per_call=None, rows_checks=1)
     assert stats["units"] == len(units) * len(steps)
+
+
+def test_static_rank_mode_tiny_and_small():
+    """Algorithm 3 as printed: kept rows in top-index order, decode cuts a prefix before attending."""
+    wl = get_workload("tiny")
+    stats = run_and_check(wl, wl.decode_steps, static_rank=1)
+    assert stats["units"] == wl.decode_steps + 1
+    wl = get_workload("tiny").scaled(dtype="bf16", head_dim=128, num_heads=3, num_layers=5, batch=2, sys_len=3,
+                                     num_visual=131, text_len_min=1, text_len_max=37, decode_steps=9,
+                                     first_prune_layer=1, stride=2, step_ratio_bp=2000, tau=9.0, num_planted=7)
+    run_and_check(wl, 9, static_rank=1)
+
+
+def test_static_rank_mode_llava15_7b():
+    wl = get_workload("llava15_7b")
+    steps = [0, 1, 2, 100, 255, 256]
+    stats = run_and_check(wl, wl.decode_steps, check_steps=steps, static_rank=1)
+    assert stats["units"] == 32 * len(steps)

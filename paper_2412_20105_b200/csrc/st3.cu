@@ -65,6 +65,10 @@ struct StepParams {
   int chunk_rows;           // rows per work item (<= the kernel's tile capacity)
   int total_work;           // work items x heads of this launch
   int first_dynamic;        // managers of the attention grid: items below this index are pre-assigned
+  unsigned counter_base;    // value of the work counter when this launch starts (it is never reset)
+  int* flags;               // [l][b] sequence number of the last finish launch that is done with (l, b)
+  int seq;                  // sequence number of this step's launches
+  int req[kMaxLayers];      // flag value the visual rows of a layer must have reached before they are read
   unsigned h_mul, h_shift;  // fast division by H
   int cvp[kMaxLayers + 1];  // prefix sum of visual chunks per layer (relative layer index)
   int lstart[kMaxLayers + 1];       // first work item of each layer: B * (cvp[l] + l * ct)
@@ -245,6 +249,33 @@ __device__ __forceinline__ bool ring_wait(uint64_t* bar, uint32_t parity, volati
   return __all_sync(0xffffffffu, ok);
 }
 
+// The finish launch of the previous step may still be running when this kernel starts (programmatic
+// dependent launch): visual rows of (l, b) are read only after that launch has signalled them.
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(int* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ bool flag_wait(const int* flag, int want, volatile int* abort_flag, int* status) {
+  bool ok = ld_acquire(flag) - want >= 0;
+  if (!ok) {
+    const long long t0 = clock64();
+    while (!(ok = ld_acquire(flag) - want >= 0)) {
+      __nanosleep(100);
+      if (*abort_flag) break;
+      if (clock64() - t0 > kWaitCycles) {
+        *abort_flag = 1;
+        atomicOr(status, ST3_DEV_COPY_TIMEOUT);
+        break;
+      }
+    }
+  }
+  return __all_sync(0xffffffffu, ok);
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const StepParams p) {
   constexpr int EPL = 16 / sizeof(T);      // elements per 16-byte chunk
@@ -294,22 +325,24 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
     // A decoded work item, held in registers until its slot is free.
     struct Dec {
       bool valid, has_new;
-      int nrows, nbulk, want_logits;
-      long long slot, lbh, oidx, glog;
+      int nrows, nbulk, want_logits, wait_for;
+      long long slot, lbh, oidx, glog, lb;
       const unsigned char *srcK, *srcV;
       T *newK, *newV;
       uint4 nv[NV];
     };
     int lcur = 0;  // layer of the previous item: this warp's items arrive in increasing order
+    long long lb_ready = -1;  // the (l, b) whose visual rows were last seen released by the previous finish launch
     // the first item of every manager is fixed (no round trip to the counter before the first copy);
     // the counter starts behind those and hands out the rest
     int x_next = (int)blockIdx.x * kSlots + s;
 
     auto decode = [&](Dec& d) {
       const int x = __shfl_sync(0xffffffffu, x_next, 0);
-      d.valid = x < total;
+      d.valid = (unsigned)x < (unsigned)total;
       if (!d.valid) return;
-      if (lane == 0) x_next = atomicAdd(p.work_counter, 1);  // prefetch the index after this one
+      if (lane == 0)  // prefetch the index after this one
+        x_next = p.first_dynamic + (int)(atomicAdd(reinterpret_cast<unsigned*>(p.work_counter), 1u) - p.counter_base);
       const int item = (int)fast_div((unsigned)x, p.h_mul, p.h_shift);
       const int h = x - item * H;
       while (lcur + 1 < p.layer_count && item >= p.lstart[lcur + 1]) ++lcur;
@@ -341,6 +374,12 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
       d.srcK = reinterpret_cast<const unsigned char*>(gK) + (size_t)r0 * ROWB;
       d.srcV = reinterpret_cast<const unsigned char*>(gV) + (size_t)r0 * ROWB;
       d.want_logits = is_vis && p.ntgt[l_rel] < p.ncur[l_rel];
+      d.lb = (long long)l * p.B + b;
+      d.wait_for = is_vis && d.lb != lb_ready ? p.req[l_rel] : 0;
+      if (d.wait_for && ld_acquire(p.flags + d.lb) - d.wait_for >= 0) {  // looked up here, off the critical path
+        d.wait_for = 0;
+        lb_ready = d.lb;
+      }
       d.glog = d.lbh * p.Nv + r0;
       d.slot = (long long)item * H + h;
       if (d.has_new) {
@@ -356,6 +395,10 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
     };
     // Starts the copies of a decoded item into this (free) slot.
     auto issue = [&](const Dec& d, int g) {  // g: the consumer group this use of the slot belongs to
+      if (d.wait_for) {
+        if (!flag_wait(p.flags + d.lb, d.wait_for, abort_flag, p.status)) return;
+        lb_ready = d.lb;
+      }
       if (d.has_new) {
         if (lane < 2 * LN) {
           const int kv = lane / LN;
@@ -580,6 +623,8 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   __shared__ float s_half[kFinishThreads / 2];
   __shared__ int s_sel[3];  // digit, count above, count in bin
 
+  // the next step's attention launch may start now; it waits on p.flags for what this launch changes
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int tid = threadIdx.x, lane = tid & 31;
   const int B = p.B, H = p.H, Nv = p.Nv;
   const int units = p.layer_count * B;  // blocks [0, units) trim, blocks [units, 2 units) write the output
@@ -639,7 +684,11 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
 
   // ===================== TRIM block =====================
   const int tt = tid, warp = tid >> 5;
-  if (blockIdx.x == 0 && tt == 0) *p.work_counter = p.first_dynamic;  // ready for the next attention launch
+  // Signals that this launch is done with the visual rows, ids and logits of (l, b).
+  auto done = [&]() {
+    __syncthreads();
+    if (tt == 0) { __threadfence(); st_release(p.flags + lb, p.seq); }
+  };
   const int n_host = p.ncur[l_rel];
   const int k = min(n_host, p.ntgt[l_rel]);
   const bool evicts = k < n_host;  // same answer in every thread
@@ -649,6 +698,7 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
       if (n_dev != p.nold[l_rel]) atomicOr(p.status, ST3_DEV_COUNT_MISMATCH);
       else if (n_host != n_dev) p.n_cur[lb] = n_host;  // static-rank cut: only the count changes
     }
+    done();
     return;
   }
   int* ids = p.ids + lb * Nv;
@@ -682,6 +732,7 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   __syncthreads();
   if (n_dev != n_host) {  // host bookkeeping and device state disagree: flag, do not touch
     if (tt == 0) atomicOr(p.status, ST3_DEV_COUNT_MISMATCH);
+    done();
     return;
   }
 
@@ -790,6 +841,7 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
     __syncthreads();  // every thread has read the old ids it needs
     for (int j = tt; j < k; j += kFinishThreads) ids[j] = s_mover[s_hole[j]];
     if (tt == 0) p.n_cur[lb] = k;
+    done();
     return;
   }
 
@@ -828,6 +880,7 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   const int nmove = total & 0xffff;
   if (nmove != (total >> 16)) {  // cannot happen when exactly k keys pass the threshold
     if (tt == 0) atomicOr(p.status, ST3_DEV_RANGE);
+    done();
     return;
   }
 
@@ -848,6 +901,7 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   if (tt < nmove) ids[s_hole[tt]] = id_moved;
   for (int j = tt + kFinishThreads; j < nmove; j += kFinishThreads) ids[s_hole[j]] = ids[s_mover[j]];
   if (tt == 0) p.n_cur[lb] = k;
+  done();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -907,7 +961,7 @@ inline void make_fast_div(unsigned d, unsigned* mul, unsigned* shift) {
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 struct Layout {
-  size_t elem, cache, part_ml, part_acc, logits, mass, ids, n_cur, text_len, status, stage_q, stage_k, stage_v,
+  size_t elem, cache, part_ml, part_acc, part_ml_bytes, part_acc_bytes, logits, mass, ids, n_cur, flags, text_len, status, stage_q, stage_k, stage_v,
       stage_o, total;
   long long lbh_stride;
   int cap_txt, chunk_rows, max_items;
@@ -959,12 +1013,17 @@ Layout make_layout(const st3_config* c) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   L.cache = take(lbh * (size_t)L.lbh_stride * L.elem);
-  L.part_ml = take((size_t)L.max_items * c->num_heads * 2 * sizeof(float));
-  L.part_acc = take((size_t)L.max_items * c->num_heads * c->head_dim * sizeof(float));
+  // two copies of the partials: a step's attention launch may run while the previous step's finish
+  // launch is still merging
+  L.part_ml_bytes = align_up((size_t)L.max_items * c->num_heads * 2 * sizeof(float), 256);
+  L.part_acc_bytes = align_up((size_t)L.max_items * c->num_heads * c->head_dim * sizeof(float), 256);
+  L.part_ml = take(2 * L.part_ml_bytes);
+  L.part_acc = take(2 * L.part_acc_bytes);
   L.logits = take(lbh * (size_t)c->num_visual * sizeof(float));
   L.mass = take(lb * (size_t)c->num_visual * sizeof(float));
   L.ids = take(lb * (size_t)c->num_visual * sizeof(int));
   L.n_cur = take(lb * sizeof(int));
+  L.flags = take(lb * sizeof(int));
   L.text_len = take((size_t)c->batch * sizeof(int));
   L.status = take(256);
   const size_t io = lbh * c->head_dim * L.elem;
@@ -1011,6 +1070,9 @@ struct st3_ctx {
   std::vector<cudaEvent_t> ev_pool;  // triples: before attend, after attend, after finish
   size_t ev_used;
   int attend_smem, finish_smem, num_sms, attend_ctas_per_sm;
+  int seq;                     // sequence number of the next step's launches (starts at 1)
+  unsigned counter_base;       // what the device work counter will read when the next launch starts
+  std::vector<int> flag_req;   // per layer: sequence number of the last finish launch over it (0: none)
 };
 
 namespace {
@@ -1038,7 +1100,21 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
     cudaEventRecord(e0, st);
   }
   (void)total_items;
-  st3_attend_kernel<T, D><<<(unsigned)(ctx->num_sms * ctx->attend_ctas_per_sm), kAttendThreads, ctx->attend_smem, st>>>(p);
+  {
+    // Programmatic dependent launch: this launch may start while the previous step's finish launch is
+    // still running (that kernel allows it at its start); p.flags orders what the two share.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(ctx->num_sms * ctx->attend_ctas_per_sm));
+    cfg.blockDim = dim3(kAttendThreads);
+    cfg.dynamicSmemBytes = (size_t)ctx->attend_smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (ctx->profiling || ingest) ? 0 : 1;
+    if (cudaLaunchKernelEx(&cfg, st3_attend_kernel<T, D>, p) != cudaSuccess) return ST3_ERR_CUDA;
+  }
   if (e1) cudaEventRecord(e1, st);
   st3_finish_kernel<T, D><<<(unsigned)(2 * p.layer_count * c.batch), kFinishThreads, ctx->finish_smem, st>>>(p);
   if (e2) cudaEventRecord(e2, st);
@@ -1073,8 +1149,11 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
   memset(&p, 0, sizeof(p));
   p.q = q; p.k_new = prefill ? nullptr : k; p.v_new = prefill ? nullptr : v; p.out = out;
   p.cache = ctx->ws + L.cache;
-  p.part_ml = reinterpret_cast<float*>(ctx->ws + L.part_ml);
-  p.part_acc = reinterpret_cast<float*>(ctx->ws + L.part_acc);
+  p.part_ml = reinterpret_cast<float*>(ctx->ws + L.part_ml + (ctx->seq & 1) * L.part_ml_bytes);
+  p.part_acc = reinterpret_cast<float*>(ctx->ws + L.part_acc + (ctx->seq & 1) * L.part_acc_bytes);
+  p.flags = reinterpret_cast<int*>(ctx->ws + L.flags);
+  p.seq = ctx->seq;
+  p.counter_base = ctx->counter_base;
   p.logits = reinterpret_cast<float*>(ctx->ws + L.logits);
   p.mass_by_id = reinterpret_cast<float*>(ctx->ws + L.mass);
   p.ids = reinterpret_cast<int*>(ctx->ws + L.ids);
@@ -1097,6 +1176,7 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
     int ncur = prefill ? c.num_visual : ctx->n_host[l];
     const int tgt = ctx->n_tab[(size_t)l * (c.max_decode_steps + 1) + step];
     p.nold[i] = ncur;
+    p.req[i] = prefill ? 0 : ctx->flag_req[l];  // prefill follows the ingest launch in stream order
     if (c.static_rank && !prefill && tgt < ncur) ncur = tgt;  // cut first, then attend (Algorithm 3)
     p.ncur[i] = ncur;
     p.ntgt[i] = tgt < ncur ? tgt : ncur;
@@ -1120,7 +1200,10 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
   for (int i = 0; i < layer_count; ++i) {
     ctx->n_host[layer_begin + i] = p.ntgt[i];
     ctx->last_step[layer_begin + i] = step;
+    ctx->flag_req[layer_begin + i] = ctx->seq;
   }
+  ctx->seq++;
+  ctx->counter_base += (unsigned)p.total_work;  // one fetch per work item (the first of each manager is fixed)
   ctx->last_stream = st;
   return ST3_OK;
 }
@@ -1165,6 +1248,9 @@ st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, 
   ctx->max_text = 0;
   ctx->last_stream = nullptr;
   ctx->launches = 0;
+  ctx->seq = 1;
+  ctx->counter_base = 0;
+  ctx->flag_req.assign(cfg->num_layers, 0);
   ctx->profiling = false;
   ctx->ev_used = 0;
   ctx->attend_smem = kSlots * (2 * tile_bytes(cfg) + kQBytes);
@@ -1183,11 +1269,7 @@ st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, 
 #undef ST3_ATTR
   if (s == ST3_OK) {
     // bookkeeping area (scores, ids, counts, text lengths, status word) starts cleared
-    // ... except the work counter, which starts behind the pre-assigned first item of every manager
-    const int first_dynamic = ctx->num_sms * ctx->attend_ctas_per_sm * kSlots;
     if (cudaMemsetAsync(ctx->ws + L.mass, 0, L.stage_q - L.mass, nullptr) != cudaSuccess ||
-        cudaMemcpyAsync(ctx->ws + L.status + 16 * sizeof(int), &first_dynamic, sizeof(int), cudaMemcpyHostToDevice,
-                        nullptr) != cudaSuccess ||
         cudaStreamSynchronize(nullptr) != cudaSuccess)
       s = ST3_ERR_CUDA;
   }

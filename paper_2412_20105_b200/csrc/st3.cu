@@ -511,8 +511,9 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
           u64 a2[CPL];
 #pragma unroll
           for (int j = 0; j < CPL; ++j) a2[j] = 0ull;
-          if (ok[g]) {
-            const unsigned char* row = sK + (size_t)r * ROWB + c4 * (CPL * 16);
+          {
+            // branch-free: a row past the end re-reads the last valid row and its logit is discarded
+            const unsigned char* row = sK + (size_t)min(r, nrows - 1) * ROWB + c4 * (CPL * 16);
 #pragma unroll
             for (int j = 0; j < CPL; ++j) {
               const int jj = (j + rot) & (CPL - 1);
@@ -555,14 +556,13 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
         const unsigned char* vrow = sV + (size_t)base * ROWB + lane * (DPL * (int)sizeof(T));
 #pragma unroll
         for (int rr = 0; rr < TR; ++rr) {
+          // branch-free: rows past the end carry probability 0 and re-read the last valid row
           const float pv = __shfl_sync(0xffffffffu, pr[rr / 8], (rr % 8) * 4);
-          if (rr < nmine) {
-            u64 v2[DPL / 2];
-            load_pairs<T, DPL>(vrow + (size_t)rr * ROWB, v2);
-            const u64 pp = pack2(pv, pv);
+          u64 v2[DPL / 2];
+          load_pairs<T, DPL>(vrow + (size_t)min(rr, nmine - 1) * ROWB, v2);
+          const u64 pp = pack2(pv, pv);
 #pragma unroll
-            for (int i = 0; i < DPL / 2; ++i) fma2(acc2[i], pp, v2[i]);
-          }
+          for (int i = 0; i < DPL / 2; ++i) fma2(acc2[i], pp, v2[i]);
         }
         // the warp's un-normalised result [D] goes over its own (consumed) K rows
         float* res = reinterpret_cast<float*>(sK + (size_t)base * ROWB) + lane * DPL;

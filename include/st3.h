@@ -153,7 +153,8 @@ st3_status st3_get_rows(st3_ctx* ctx, int32_t layer, int32_t b, int32_t h, void*
                         void* k_txt, void* v_txt, void* cuda_stream);
 
 /* Synchronises the stream last used by this context and returns the device status word through
- * *word (host).  Returns ST3_ERR_DEVICE_CHECK if it is non-zero. */
+ * *word (host).  Returns ST3_ERR_DEVICE_CHECK if it is non-zero; the word is sticky and the results of
+ * a context that has reported one are undefined from then on: destroy it and create a new one. */
 st3_status st3_get_status(st3_ctx* ctx, int32_t* word);
 
 /* Visual + non-visual K/V rows currently held, summed over layers and sequences (host

@@ -156,3 +156,72 @@ def test_layer_by_layer_calls_match_one_call_for_all_layers():
         assert a.ctx.status() == 0 and b.ctx.status() == 0
     finally:
         a.close(); b.close()
+
+
+def _handmade(nv, H=2, D=64, sys_len=2, text=3, steps=4, keep_bp=5000, **cfg_kw):
+    cfg = B.make_config(num_layers=1, num_heads=H, head_dim=D, dtype="f32", batch=1, sys_len=sys_len,
+                        num_visual=nv, max_text_len=text, max_decode_steps=steps, stride=1, step_ratio_bp=0,
+                        first_prune_layer=0, first_ratio_bp=10000 - keep_bp, tau=float(steps), **cfg_kw)
+    return cfg, B.Context(cfg)
+
+
+@pytest.mark.parametrize("static_rank", [0, 1])
+def test_equal_scores_keep_the_lowest_original_indices(static_rank):
+    """Every visual key identical => every visual score identical: Top must fall back on the index."""
+    nv, H, D, sys_len, text = 200, 2, 64, 2, 3
+    cfg, ctx = _handmade(nv, H, D, sys_len, text, static_rank=static_rank)
+    try:
+        g = torch.Generator().manual_seed(5)
+        T0 = sys_len + nv + text
+        K = torch.randn(1, 1, H, T0, D, generator=g)
+        V = torch.randn(1, 1, H, T0, D, generator=g)
+        K[:, :, :, sys_len:sys_len + nv] = K[:, :, :, sys_len:sys_len + 1]          # all visual keys alike
+        q = torch.randn(1, 1, H, D, generator=g)
+        out = torch.empty(1, 1, H, D, device="cuda")
+        ctx.prefill_select(q.cuda(), K.cuda(), V.cuda(), [text], out)
+        ids, cnt, mass = ctx.get_kept(0)
+        n = int(cnt[0])
+        assert n == nv // 2
+        assert sorted(ids[0, :n].tolist()) == list(range(n))                        # the n lowest indices
+        if static_rank:
+            assert ids[0, :n].tolist() == list(range(n))                            # and in index order
+        m = mass[0].cpu().numpy()
+        assert np.all(m == m[0]) and m[0] > 0                                       # bit-identical scores
+        # decode steps keep dropping the highest remaining indices
+        for t in range(1, 4):
+            kn = torch.randn(1, 1, H, D, generator=g).cuda()
+            ctx.decode_step(t, q.cuda(), kn, kn, out)
+            ids, cnt, _ = ctx.get_kept(0)
+            k = B.st3_schedule_count(cfg, 0, t)
+            assert int(cnt[0]) == k and sorted(ids[0, :k].tolist()) == list(range(k))
+        assert ctx.status() == 0
+    finally:
+        ctx.close()
+
+
+def test_two_score_levels_with_ties_at_the_cut():
+    """Half of the visual keys get a clearly larger logit; the cut falls inside the lower tie class."""
+    nv, H, D, sys_len, text = 96, 2, 64, 1, 2
+    cfg, ctx = _handmade(nv, H, D, sys_len, text, keep_bp=7500)
+    try:
+        g = torch.Generator().manual_seed(6)
+        T0 = sys_len + nv + text
+        K = torch.randn(1, 1, H, T0, D, generator=g)
+        V = torch.randn(1, 1, H, T0, D, generator=g)
+        q = torch.randn(1, 1, H, D, generator=g)
+        lo, hi = K[:, :, :, sys_len:sys_len + 1].clone(), None
+        hi = lo + 0.5 * q[:, :, :, None, :]                                          # larger q.k for every head
+        strong = torch.zeros(nv, dtype=torch.bool)
+        strong[torch.randperm(nv, generator=g)[:nv // 2]] = True
+        K[:, :, :, sys_len:sys_len + nv] = torch.where(strong[None, None, None, :, None], hi, lo)
+        out = torch.empty(1, 1, H, D, device="cuda")
+        ctx.prefill_select(q.cuda(), K.cuda(), V.cuda(), [text], out)
+        ids, cnt, _ = ctx.get_kept(0)
+        n = int(cnt[0])
+        assert n == 72
+        weak_ids = [i for i in range(nv) if not strong[i]]
+        want = set(i for i in range(nv) if strong[i]) | set(weak_ids[:72 - 48])      # all strong + lowest weak
+        assert set(ids[0, :n].tolist()) == want
+        assert ctx.status() == 0
+    finally:
+        ctx.close()

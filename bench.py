@@ -198,6 +198,48 @@ class Job:
             if rc:
                 raise B.St3Error(rc, f"st3_decode_step t={t}")
 
+    def prefill_only(self):
+        self.B.st3_prefill_select(self.ctx.handle, 0, self.wl.num_layers, self.q0.data_ptr(), self.K.data_ptr(),
+                                  self.V.data_ptr(), self.text, self.out0.data_ptr(), self.stream)
+
+    def generation_per_layer(self):
+        """The calling pattern of a real model: one call per layer, prefill and every decode step."""
+        B, h, L, st = self.B, self.ctx.handle, self.wl.num_layers, self.stream
+        lb0 = self.q0[0].numel() * self.q0.element_size()                 # bytes of one layer of q / out
+        kvb = self.K[0].numel() * self.K.element_size()
+        for l in range(L):
+            B.st3_prefill_select(h, l, 1, self.q0.data_ptr() + l * lb0, self.K.data_ptr() + l * kvb,
+                                 self.V.data_ptr() + l * kvb, self.text, self.out0.data_ptr() + l * lb0, st)
+        q, k, v, o, nb = self.q.data_ptr(), self.kn.data_ptr(), self.vn.data_ptr(), self.out.data_ptr(), self.io_bytes
+        step_fn = self.lib.st3_decode_step
+        for t in range(1, self.wl.decode_steps + 1):
+            off = (t - 1) * nb
+            for l in range(L):
+                o2 = off + l * lb0
+                rc = step_fn(h, t, l, 1, q + o2, k + o2, v + o2, o + o2, st)
+                if rc:
+                    raise B.St3Error(rc, f"st3_decode_step t={t} l={l}")
+
+    def rows_held_curve(self, points=9):
+        """(step, visual rows, other rows, K/V bytes held) along one generation: host bookkeeping."""
+        wl, B, h = self.wl, self.B, self.ctx.handle
+        e = 2 if wl.dtype == "bf16" else 4
+        row_bytes = 2 * wl.num_heads * wl.head_dim * e
+        want = sorted(set(int(round(x)) for x in np.linspace(0, wl.decode_steps, points)))
+        self.prefill_only()
+        out = []
+        q, k, v, o, nb = self.q.data_ptr(), self.kn.data_ptr(), self.vn.data_ptr(), self.out.data_ptr(), self.io_bytes
+        for t in range(0, wl.decode_steps + 1):
+            if t:
+                off = (t - 1) * nb
+                B.st3_decode_step(h, t, 0, wl.num_layers, q + off, k + off, v + off, o + off, self.stream)
+            if t in want:
+                vis, oth = B.st3_rows_held(h)
+                full = wl.batch * wl.num_layers * wl.num_visual
+                out.append({"step": t, "visual_rows": vis, "other_rows": oth, "kv_bytes": (vis + oth) * row_bytes,
+                            "kv_bytes_untrimmed": (full + oth) * row_bytes})
+        return out
+
     def make_host(self):
         self.hK, self.hV = self.K.cpu().pin_memory(), self.V.cpu().pin_memory()
         self.hq0 = self.q0.cpu().pin_memory()
@@ -428,6 +470,14 @@ def main():
         line["static_rank"] = {"value": tokens_per_gen * args.steps / (ms_stat * 1e-3), "unit": UNIT}
         stat.ctx.close()
         del stat
+        # prefill-select alone, the one-call-per-layer pattern, and K/V held along a generation
+        ms_pre = timed(job.prefill_only, args.steps, False)
+        line["prefill_select_ms"] = ms_pre / args.steps
+        job.generation_per_layer()
+        ms_pl = timed(job.generation_per_layer, max(1, args.steps // 2), False)
+        job.ctx.status()
+        line["per_layer_calls"] = {"value": tokens_per_gen * max(1, args.steps // 2) / (ms_pl * 1e-3), "unit": UNIT}
+        line["kv_held"] = job.rows_held_curve()
         # the oracle on the host cores, bounded sample
         ns = 24 if wl.batch == 1 else max(1, 24 // wl.batch)
         K, V, q0 = job.K.cpu(), job.V.cpu(), job.q0.cpu()

@@ -213,6 +213,34 @@ def prefill_select(q_last, K, V, sys_len: int, num_visual: int, n_keep: int, ran
     return out, mass, cache
 
 
+def prefill_select_scored(q_last, K, V, sys_len: int, num_visual: int, n_keep: int, scores,
+                          rank_ordered: bool = False):
+    """Prefill of one (sequence, layer) the way Algorithm 1 / Eq. 3 word it: the visual tokens are
+    pruned BEFORE the layer runs, by scores that come from outside (the previous layer's alpha),
+    and the layer then attends over [S | kept V | I] only.
+    Returns (out [H, D], cache).
+    """
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    scores = np.asarray(scores, dtype=np.float64)
+    ids_all = np.arange(num_visual, dtype=np.int64)
+    if rank_ordered:
+        kept = rank_order(scores, ids_all)[:max(0, min(int(n_keep), num_visual))]
+    else:
+        kept = select_top(scores, ids_all, n_keep)
+    v0, v1 = sys_len, sys_len + num_visual
+    cache = LayerCache(
+        K_sys=K[:, :v0].copy(), V_sys=V[:, :v0].copy(),
+        K_vis=K[:, v0:v1][:, kept].copy(), V_vis=V[:, v0:v1][:, kept].copy(),
+        ids=ids_all[kept].copy(),
+        K_txt=K[:, v1:].copy(), V_txt=V[:, v1:].copy(),
+        last_mass=scores,
+    )
+    Kc, Vc = cache.rows()
+    out, _ = attend(q_last, Kc, Vc)
+    return out, cache
+
+
 def decode_step(cache: LayerCache, q, k_new, v_new, n_target: int):
     """Decode half of Algorithm 3 with Eq. 7 for one (sequence, layer), one step.
 

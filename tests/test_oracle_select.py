@@ -109,3 +109,27 @@ def test_static_rank_decode_truncates_the_saved_order():
     assert np.allclose(o, attend(q, Kx, Vx)[0], rtol=1e-13, atol=1e-15)
     decode_step_static(c, q, kn, vn, 9)                           # never grows
     assert c.n_cur == 5
+
+
+def test_externally_scored_prefill_prunes_before_it_attends():
+    from oracle.st3_oracle import prefill_select_scored, attend
+    r = np.random.default_rng(23)
+    H, D, sys_len, nv, text = 2, 4, 2, 11, 3
+    T0 = sys_len + nv + text
+    K, V = r.standard_normal((H, T0, D)), r.standard_normal((H, T0, D))
+    q = r.standard_normal((H, D))
+    scores = r.permutation(nv).astype(np.float64)                  # distinct: top-5 = the 5 largest
+    out, c = prefill_select_scored(q, K, V, sys_len, nv, 5, scores)
+    want = np.sort(np.argsort(-scores)[:5])
+    assert np.array_equal(c.ids, want)
+    rows = list(range(sys_len)) + (sys_len + want).tolist() + list(range(sys_len + nv, T0))
+    assert np.allclose(out, attend(q, K[:, rows], V[:, rows])[0], rtol=1e-13, atol=1e-15)
+    # keeping everything reduces to plain attention over the whole prompt
+    out_all, c_all = prefill_select_scored(q, K, V, sys_len, nv, nv, scores)
+    assert np.allclose(out_all, attend(q, K, V)[0], rtol=1e-13, atol=1e-15) and c_all.n_cur == nv
+    # fed with the layer's own scores it keeps what prefill_select keeps
+    o_self, m_self, c_self = prefill_select(q, K, V, sys_len, nv, 5)
+    _, c_fed = prefill_select_scored(q, K, V, sys_len, nv, 5, m_self)
+    assert np.array_equal(c_fed.ids, c_self.ids)
+    _, c_rank = prefill_select_scored(q, K, V, sys_len, nv, 5, scores, rank_ordered=True)
+    assert c_rank.ids.tolist() == np.argsort(-scores)[:5].tolist()

@@ -122,6 +122,17 @@ st3_status st3_prefill_select(st3_ctx* ctx, int32_t layer_begin, int32_t layer_c
                               const void* q_last, const void* k, const void* v,
                               const int32_t* text_len, void* out, void* cuda_stream);
 
+/* Prefill as Algorithm 1 and Eq. 3 word it: the visual tokens of each layer are pruned BEFORE the
+ * layer runs, by scores that come from outside (the previous layer's alpha), and the layer then
+ * attends over [S | kept V | I] only.  Same arguments as st3_prefill_select plus
+ *   scores   dev  [layer_count][B][num_visual] fp32, any finite values, indexed by original visual
+ *                 index; the n(l,0) largest are kept (ties toward the lower index)
+ * st3_get_kept's mass then returns these scores. */
+st3_status st3_prefill_select_scored(st3_ctx* ctx, int32_t layer_begin, int32_t layer_count,
+                                     const void* q_last, const void* k, const void* v,
+                                     const int32_t* text_len, const float* scores, void* out,
+                                     void* cuda_stream);
+
 /* One decode step (Algorithm 3's decode half with Eq. 7) for the given layers: append, attend,
  * score, select, compact.  `step` counts from 1 and must be the previous step of each of these
  * layers plus one (else ST3_ERR_BAD_STATE); step > max_decode_steps gives ST3_ERR_CAPACITY.

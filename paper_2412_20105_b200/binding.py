@@ -19,7 +19,8 @@ ST3_F32, ST3_BF16 = 0, 1
 ST3_ANNEAL_COSINE, ST3_ANNEAL_NONE, ST3_ANNEAL_LINEAR, ST3_ANNEAL_EXP = 0, 1, 2, 3
 DEV_COUNT_MISMATCH, DEV_NONFINITE, DEV_COPY_TIMEOUT, DEV_RANGE = 1, 2, 4, 8
 
-EXPORTS = ["st3_schedule_count", "st3_workspace_size", "st3_create", "st3_prefill_select", "st3_decode_step",
+EXPORTS = ["st3_schedule_count", "st3_workspace_size", "st3_create", "st3_prefill_select",
+           "st3_prefill_select_scored", "st3_decode_step",
            "st3_decode_step_host", "st3_get_kept", "st3_get_rows", "st3_get_status", "st3_rows_held",
            "st3_profile_enable", "st3_profile_read", "st3_launch_count", "st3_status_string", "st3_destroy",
            "st3_attend_noalloc"]
@@ -59,6 +60,7 @@ def load():
     lib.st3_workspace_size.argtypes = [cfgp, C.POINTER(C.c_size_t)]
     lib.st3_create.argtypes = [cfgp, vp, C.c_size_t, C.POINTER(vp)]
     lib.st3_prefill_select.argtypes = [vp, i32, i32, vp, vp, vp, C.POINTER(i32), vp, vp]
+    lib.st3_prefill_select_scored.argtypes = [vp, i32, i32, vp, vp, vp, C.POINTER(i32), vp, vp, vp]
     lib.st3_decode_step.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.st3_decode_step_host.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.st3_get_kept.argtypes = [vp, i32, vp, vp, vp, vp]
@@ -116,6 +118,14 @@ def st3_prefill_select(ctx, layer_begin, layer_count, q_last, k, v, text_len, ou
     arr = (C.c_int32 * len(text_len))(*[int(x) for x in text_len])
     _check(load().st3_prefill_select(ctx, layer_begin, layer_count, q_last, k, v, arr, out, stream),
            "st3_prefill_select")
+
+
+def st3_prefill_select_scored(ctx, layer_begin, layer_count, q_last, k, v, text_len, scores, out, stream=0):
+    """As st3_prefill_select, but the kept set comes from `scores` (device address, fp32
+    [layer_count][B][num_visual]) and the layer attends over the kept rows only."""
+    arr = (C.c_int32 * len(text_len))(*[int(x) for x in text_len])
+    _check(load().st3_prefill_select_scored(ctx, layer_begin, layer_count, q_last, k, v, arr, scores, out, stream),
+           "st3_prefill_select_scored")
 
 
 def st3_decode_step(ctx, step, layer_begin, layer_count, q, k_new, v_new, out, stream=0):
@@ -219,6 +229,11 @@ class Context:
     def prefill_select(self, q_last, k, v, text_len, out, layer_begin=0):
         st3_prefill_select(self.handle, layer_begin, q_last.shape[0], self._ptr(q_last), self._ptr(k), self._ptr(v),
                            text_len, self._ptr(out), self._stream())
+
+    def prefill_select_scored(self, q_last, k, v, text_len, scores, out, layer_begin=0):
+        assert scores.is_cuda and scores.is_contiguous() and scores.dtype == self.torch.float32
+        st3_prefill_select_scored(self.handle, layer_begin, q_last.shape[0], self._ptr(q_last), self._ptr(k),
+                                  self._ptr(v), text_len, scores.data_ptr(), self._ptr(out), self._stream())
 
     def decode_step(self, step, q, k_new, v_new, out, layer_begin=0):
         st3_decode_step(self.handle, step, layer_begin, q.shape[0], self._ptr(q), self._ptr(k_new), self._ptr(v_new),

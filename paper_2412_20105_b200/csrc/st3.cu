@@ -82,6 +82,7 @@ struct StepParams {
   const void* v_in;
   int t0_max;
   int static_rank;          // 1: keep the kept rows in top-index order, cut them without scoring
+  const float* ext_scores;  // prefill with the caller's scores [layer_count][B][Nv]: selection only, no merge
 };
 
 // ------------------------------------------------------------------------------------------
@@ -638,6 +639,7 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   const float2* ml = reinterpret_cast<const float2*>(p.part_ml);
 
   if (out_role) {
+    if (p.ext_scores) return;  // selection-only launch: nothing to merge yet
     // ===================== OUT block: attention output of every head =====================
     constexpr int kMergeBatch = 8;  // partials in flight per round trip
     for (int h = tid >> 5; h < H; h += kFinishWarps) {
@@ -716,18 +718,21 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   const int ri = tt % kRowsPerPass, hg = tt / kRowsPerPass;
   float pre[kHeadBatch];
   int id0 = 0;
-  if (ri < n_cur) {
-    if (hg == 0) id0 = ids[ri];
+  const bool own_scores = p.ext_scores == nullptr;
+  if (own_scores) {
+    if (ri < n_cur) {
+      if (hg == 0) id0 = ids[ri];
 #pragma unroll
-    for (int j = 0; j < kHeadBatch; ++j) {
-      const int h = hg * kHeadBatch + j;
-      pre[j] = h < H ? logits[(long long)h * Nv + ri] : -INFINITY;
+      for (int j = 0; j < kHeadBatch; ++j) {
+        const int h = hg * kHeadBatch + j;
+        pre[j] = h < H ? logits[(long long)h * Nv + ri] : -INFINITY;
+      }
     }
-  }
-  for (int h = warp; h < H; h += kFinishWarps) {
-    float M, Lh;
-    merge_stats(ml, item0, nit, H, h, lane, M, Lh);
-    if (lane == 0) { s_M[h] = M; s_invL[h] = 1.f / Lh; }
+    for (int h = warp; h < H; h += kFinishWarps) {
+      float M, Lh;
+      merge_stats(ml, item0, nit, H, h, lane, M, Lh);
+      if (lane == 0) { s_M[h] = M; s_invL[h] = 1.f / Lh; }
+    }
   }
   __syncthreads();
   if (n_dev != n_host) {  // host bookkeeping and device state disagree: flag, do not touch
@@ -738,7 +743,21 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
 
   // ---- visual scores: probability of every visual row summed over heads ----
   bool bad = false;
-  for (int i0 = 0; i0 < n_cur; i0 += kRowsPerPass) {
+  if (!own_scores) {
+    // scores supplied by the caller (any finite float): order-preserving map of the bits to unsigned
+    const float* ext = p.ext_scores + ((long long)l_rel * B + b) * Nv;
+    for (int i = tt; i < n_cur; i += kFinishThreads) {
+      const int id = ids[i];
+      float sc = ext[id];
+      if (!(fabsf(sc) <= 3.0e38f)) { bad = true; sc = -3.0e38f; }
+      mass_by_id[id] = sc;
+      unsigned u = __float_as_uint(sc);
+      u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+      s_key[i] = ((unsigned long long)u << 32) | (unsigned long long)(0xffffffffu - (unsigned)id);
+    }
+    __syncthreads();
+  }
+  for (int i0 = 0; own_scores && i0 < n_cur; i0 += kRowsPerPass) {
     const int i = i0 + ri;
     float pm = 0.f;
     int id = id0;
@@ -1079,13 +1098,18 @@ namespace {
 
 template <typename T, int D>
 st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cudaStream_t st, const void* pk,
-                         const void* pv, bool ingest) {
+                         const void* pv, bool ingest, const StepParams* select_first) {
   const st3_config& c = ctx->cfg;
   if (ingest) {
     dim3 grid(8, (unsigned)(c.num_heads * c.batch * p.layer_count));
     st3_ingest_kernel<T, D><<<grid, kThreads, 0, st>>>(p, reinterpret_cast<const T*>(pk),
                                                        reinterpret_cast<const T*>(pv),
                                                        c.sys_len + c.num_visual + c.max_text_len);
+    ctx->launches++;
+  }
+  if (select_first) {  // prune by the caller's scores before the layer attends
+    st3_finish_kernel<T, D><<<(unsigned)(2 * p.layer_count * c.batch), kFinishThreads, ctx->finish_smem, st>>>(
+        *select_first);
     ctx->launches++;
   }
   cudaEvent_t e0 = nullptr, e1 = nullptr, e2 = nullptr;
@@ -1142,7 +1166,7 @@ bool aligned16(const void* p) { return p && (reinterpret_cast<uintptr_t>(p) & 15
 
 // Common body of prefill (step 0, ingest, no append) and decode (step >= 1, append).
 st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, const void* q, const void* k,
-                    const void* v, void* out, cudaStream_t st, bool prefill) {
+                    const void* v, void* out, cudaStream_t st, bool prefill, const float* ext_scores = nullptr) {
   const st3_config& c = ctx->cfg;
   const Layout& L = ctx->lay;
   StepParams p;
@@ -1175,6 +1199,7 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
     const int l = layer_begin + i;
     int ncur = prefill ? c.num_visual : ctx->n_host[l];
     const int tgt = ctx->n_tab[(size_t)l * (c.max_decode_steps + 1) + step];
+    if (ext_scores && tgt < ncur) ncur = tgt;  // already pruned by the selection launch when the layer attends
     p.nold[i] = ncur;
     p.req[i] = prefill ? 0 : ctx->flag_req[l];  // prefill follows the ingest launch in stream order
     if (c.static_rank && !prefill && tgt < ncur) ncur = tgt;  // cut first, then attend (Algorithm 3)
@@ -1193,7 +1218,16 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
   p.total_work = (int)(total_items * c.num_heads);
   p.first_dynamic = ctx->num_sms * ctx->attend_ctas_per_sm * kSlots;
 
-#define ST3_LAUNCH(T, D) launch_step_t<T, D>(ctx, p, (int)total_items, st, k, v, prefill)
+  StepParams psel;
+  if (ext_scores) {  // parameters of the selection-only launch: all Nv rows held, cut to the schedule
+    psel = p;
+    psel.ext_scores = ext_scores;
+    for (int i = 0; i < layer_count; ++i) {
+      psel.ncur[i] = psel.nold[i] = c.num_visual;
+      psel.ntgt[i] = p.ncur[i];
+    }
+  }
+#define ST3_LAUNCH(T, D) launch_step_t<T, D>(ctx, p, (int)total_items, st, k, v, prefill, ext_scores ? &psel : nullptr)
   const st3_status s = ST3_DISPATCH(ctx, ST3_LAUNCH);
 #undef ST3_LAUNCH
   if (s != ST3_OK) return s;
@@ -1278,9 +1312,9 @@ st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, 
   return ST3_OK;
 }
 
-st3_status st3_prefill_select(st3_ctx* ctx, int32_t layer_begin, int32_t layer_count, const void* q_last,
-                              const void* k, const void* v, const int32_t* text_len, void* out,
-                              void* cuda_stream) {
+static st3_status prefill_common(st3_ctx* ctx, int32_t layer_begin, int32_t layer_count, const void* q_last,
+                                 const void* k, const void* v, const int32_t* text_len, const float* scores,
+                                 void* out, void* cuda_stream) {
   if (!ctx || !text_len) return ST3_ERR_INVALID_ARG;
   const st3_config& c = ctx->cfg;
   if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c.num_layers) return ST3_ERR_INVALID_ARG;
@@ -1305,7 +1339,20 @@ st3_status st3_prefill_select(st3_ctx* ctx, int32_t layer_begin, int32_t layer_c
                         cudaMemcpyHostToDevice, st) != cudaSuccess)
       return ST3_ERR_CUDA;
   }
-  return run_step(ctx, 0, layer_begin, layer_count, q_last, k, v, out, st, true);
+  return run_step(ctx, 0, layer_begin, layer_count, q_last, k, v, out, st, true, scores);
+}
+
+st3_status st3_prefill_select(st3_ctx* ctx, int32_t layer_begin, int32_t layer_count, const void* q_last,
+                              const void* k, const void* v, const int32_t* text_len, void* out,
+                              void* cuda_stream) {
+  return prefill_common(ctx, layer_begin, layer_count, q_last, k, v, text_len, nullptr, out, cuda_stream);
+}
+
+st3_status st3_prefill_select_scored(st3_ctx* ctx, int32_t layer_begin, int32_t layer_count, const void* q_last,
+                                     const void* k, const void* v, const int32_t* text_len, const float* scores,
+                                     void* out, void* cuda_stream) {
+  if (!aligned16(scores)) return ST3_ERR_INVALID_ARG;
+  return prefill_common(ctx, layer_begin, layer_count, q_last, k, v, text_len, scores, out, cuda_stream);
 }
 
 st3_status st3_decode_step(st3_ctx* ctx, int32_t step, int32_t layer_begin, int32_t layer_count, const void* q,

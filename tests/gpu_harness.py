@@ -71,6 +71,36 @@ class GpuRun:
         self.q_cur = q0
         return self.out
 
+    def prefill_scored(self, scores):
+        """Prefill with caller-supplied scores [L, B, Nv] (prune, then attend), all layers in one call."""
+        g = self.g
+        q0 = g.queries([0], device=self.dev)[0]
+        K, V = g.prompt_kv(range(self.L), device=self.dev)
+        self.ctx.prefill_select_scored(q0, K, V, g.text_len.tolist(), scores, self.out)
+        self.q_cur = q0
+        return self.out
+
+    def check_prefill_scored_unit(self, b, l, scores):
+        wl, g, s = self.wl, self.g, self.sched
+        t0 = wl.sys_len + wl.num_visual + int(g.text_len[b])
+        K, V = g.kv_rows([b], [l], range(t0))
+        q = g.queries([0], [l])[0, 0, b]
+        sc = scores[l, b].double().cpu().numpy()
+        ref_out, cache = O.prefill_select_scored(f64(q), f64(K[0, 0]), f64(V[0, 0]), wl.sys_len, wl.num_visual,
+                                                 s.n0(l), sc, rank_ordered=self.static)
+        assert_out_close(f64(self.out[l, b]), ref_out, wl.dtype, f"scored prefill out b={b} l={l}")
+        ids, cnt, mass = self.kept(l)
+        n = int(cnt[b])
+        assert n == s.n0(l)
+        if self.static and n < wl.num_visual:     # layers that are not pruned keep the prompt's order
+            assert ids[b, :n].tolist() == cache.ids.tolist()
+        else:
+            assert sorted(ids[b, :n].tolist()) == sorted(cache.ids.tolist())
+        if n < wl.num_visual:
+            assert np.array_equal(mass[b], scores[l, b].cpu().numpy())
+        self.stats["exact"] += 1
+        self.stats["units"] += 1
+
     def inputs(self, step):
         g = self.g
         q = g.queries([step], device=self.dev)[0]

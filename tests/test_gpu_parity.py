@@ -98,3 +98,30 @@ def test_static_rank_mode_llava15_7b():
     steps = [0, 1, 2, 100, 255, 256]
     stats = run_and_check(wl, wl.decode_steps, check_steps=steps, static_rank=1)
     assert stats["units"] == 32 * len(steps)
+
+
+@pytest.mark.parametrize("static_rank", [0, 1])
+def test_prefill_with_external_scores_then_decode(static_rank):
+    """Algorithm 1's order: prune by scores from outside (the previous layer's alpha), then attend."""
+    wl = get_workload("tiny").scaled(dtype="bf16", head_dim=128, num_heads=4, num_layers=6, batch=3, sys_len=4,
+                                     num_visual=300, text_len_min=2, text_len_max=30, decode_steps=8,
+                                     first_prune_layer=2, stride=2, step_ratio_bp=1500, tau=8.0, num_planted=9)
+    run = GpuRun(wl, static_rank=static_rank)
+    try:
+        g = torch.Generator().manual_seed(7)
+        scores = torch.randn(wl.num_layers, wl.batch, wl.num_visual, generator=g).cuda()     # negatives included
+        scores[1, 0, 5] = scores[1, 0, 17]                                                   # an exact tie
+        run.prefill_scored(scores)
+        for l in range(wl.num_layers):
+            for b in range(wl.batch):
+                run.check_prefill_scored_unit(b, l, scores)
+                run.check_rows_unit(b, l, (l + b) % wl.num_heads, 0)
+        for t in range(1, 5):                                    # decode goes on from the externally chosen set
+            before = run.snapshot(range(wl.num_layers))
+            run.decode(t)
+            for l in range(wl.num_layers):
+                for b in range(wl.batch):
+                    run.check_decode_unit(b, l, t, before[l])
+        assert run.ctx.status() == 0
+    finally:
+        run.close()

@@ -183,7 +183,8 @@ def rank_order(scores: np.ndarray, ids: np.ndarray) -> np.ndarray:
     return np.lexsort((np.asarray(ids), -np.asarray(scores, dtype=np.float64)))
 
 
-def prefill_select(q_last, K, V, sys_len: int, num_visual: int, n_keep: int, rank_ordered: bool = False):
+def prefill_select(q_last, K, V, sys_len: int, num_visual: int, n_keep: int, rank_ordered: bool = False,
+                   select_scores=None):
     """Prefill half of Algorithm 3 for one (sequence, layer).
 
     K, V [H, T0, D] hold the prompt rows [S | V | I]; q_last [H, D] is the last
@@ -191,17 +192,20 @@ def prefill_select(q_last, K, V, sys_len: int, num_visual: int, n_keep: int, ran
     tokens, keeps the n_keep best (Eq. 3) and builds the cache.
     With rank_ordered the kept rows are stored in the order of the top-index list (best first),
     which is what the static-rank decode of Algorithm 3 truncates.
+    select_scores [num_visual], if given, replaces this layer's own scores in the selection: the
+    layers between two pruning layers reuse the pruning layer's choice (Sec. 3.2, strided pruning).
     Returns (out [H, D], mass [num_visual], cache).
     """
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
     out, p = attend(q_last, K, V)
     mass = visual_mass(p, sys_len, num_visual)
+    sel = mass if select_scores is None else np.asarray(select_scores, dtype=np.float64)
     ids_all = np.arange(num_visual, dtype=np.int64)
     if rank_ordered:
-        kept = rank_order(mass, ids_all)[:max(0, min(int(n_keep), num_visual))]
+        kept = rank_order(sel, ids_all)[:max(0, min(int(n_keep), num_visual))]
     else:
-        kept = select_top(mass, ids_all, n_keep)
+        kept = select_top(sel, ids_all, n_keep)
     v0, v1 = sys_len, sys_len + num_visual
     cache = LayerCache(
         K_sys=K[:, :v0].copy(), V_sys=V[:, :v0].copy(),
@@ -241,12 +245,14 @@ def prefill_select_scored(q_last, K, V, sys_len: int, num_visual: int, n_keep: i
     return out, cache
 
 
-def decode_step(cache: LayerCache, q, k_new, v_new, n_target: int):
+def decode_step(cache: LayerCache, q, k_new, v_new, n_target: int, select_scores=None):
     """Decode half of Algorithm 3 with Eq. 7 for one (sequence, layer), one step.
 
     Appends the new token's key/value, attends over every cached row, scores
     the current visual rows and, if the schedule asks for fewer rows than are
     held, keeps the n_target best and evicts the rest.
+    select_scores (one per visual row held, in cache order), if given, replaces this layer's own
+    scores in the selection (a layer that follows its stage's pruning layer).
     Returns (out [H, D], mass over the visual rows held BEFORE the eviction,
     ids held before the eviction).
     """
@@ -261,7 +267,8 @@ def decode_step(cache: LayerCache, q, k_new, v_new, n_target: int):
     ids_before = cache.ids.copy()
     n_new = min(n_cur, int(n_target))
     if n_new < n_cur:
-        kept = select_top(mass, cache.ids, n_new)
+        kept = select_top(mass if select_scores is None else np.asarray(select_scores, dtype=np.float64),
+                          cache.ids, n_new)
         cache.K_vis = cache.K_vis[:, kept]
         cache.V_vis = cache.V_vis[:, kept]
         cache.ids = cache.ids[kept]

@@ -133,3 +133,23 @@ def test_externally_scored_prefill_prunes_before_it_attends():
     assert np.array_equal(c_fed.ids, c_self.ids)
     _, c_rank = prefill_select_scored(q, K, V, sys_len, nv, 5, scores, rank_ordered=True)
     assert c_rank.ids.tolist() == np.argsort(-scores)[:5].tolist()
+
+
+def test_follower_layers_adopt_the_pruning_layers_choice():
+    """select_scores: a layer between two pruning layers keeps what the pruning layer's scores keep."""
+    r = np.random.default_rng(24)
+    H, D, sys_len, nv, text = 2, 4, 1, 9, 2
+    T0 = sys_len + nv + text
+    mk = lambda: (r.standard_normal((H, D)), r.standard_normal((H, T0, D)), r.standard_normal((H, T0, D)))
+    qa, Ka, Va = mk()
+    qb, Kb, Vb = mk()
+    oa, ma, ca = prefill_select(qa, Ka, Va, sys_len, nv, 5)
+    ob, mb, cb = prefill_select(qb, Kb, Vb, sys_len, nv, 5, select_scores=ma)
+    assert np.array_equal(ca.ids, cb.ids)                                  # same tokens ...
+    assert np.array_equal(cb.K_vis, Kb[:, sys_len + cb.ids])               # ... of the follower's own rows
+    ob_own, mb_own, _ = prefill_select(qb, Kb, Vb, sys_len, nv, 5)
+    assert np.array_equal(ob, ob_own) and np.array_equal(mb, mb_own)       # attention itself is unchanged
+    kn, vn = r.standard_normal((H, D)), r.standard_normal((H, D))
+    _, m1, _ = decode_step(ca, r.standard_normal((H, D)), kn, vn, 3)
+    decode_step(cb, r.standard_normal((H, D)), kn, vn, 3, select_scores=m1)
+    assert np.array_equal(ca.ids, cb.ids)

@@ -82,6 +82,8 @@ typedef struct {
   int32_t disable_trim;      /* 1: same kernels, nothing is ever evicted (full-KV comparison)   */
   int32_t rows_per_chunk;    /* cache rows of one work item of the attention kernel; 0 = choose  */
   int32_t static_rank;       /* 1: Algorithm 3 as printed, see below; 0: re-rank at every step   */
+  int32_t stage_shared;      /* 1: the layers between two pruning layers keep the pruning layer's */
+                             /*    choice (Sec. 3.2, strided pruning); 0: every layer chooses     */
   double tau;                /* Eq. 8: beta = cos(t*pi/(2 tau)) for t < tau, else 0             */
   double sigma;              /* only ST3_ANNEAL_EXP: beta = exp(-t/sigma)                       */
 } st3_config;
@@ -92,6 +94,11 @@ typedef struct {
  * (T' = T[l][:n], C = C[T']: no scoring, no selection, no row moves) and then attends.  With
  * static_rank = 0 (default) every step attends first and then re-ranks the held rows by the current
  * query's scores. */
+
+/* stage_shared = 1: pruning layers are first, first+S, ...; a layer between two of them evicts
+ * exactly the tokens its pruning layer evicts (decided by the pruning layer's scores), so all layers
+ * of a stage hold the same visual tokens in the same order.  Within one step the pruning layer must be
+ * processed before (or in the same call as) the layers that follow it, else ST3_ERR_BAD_STATE. */
 
 /* Scheduled visual-row count n(l, t) of layer `layer` after decode step `step` (0 = after
  * prefill).  Pure host function.  PVTP: layers below first_prune_layer keep everything; layer l

@@ -51,7 +51,9 @@ struct StepParams {
   void* cache;
   float* part_ml;        // [item*H + h][2]  (m, l) in the log2 domain
   float* part_acc;       // [item*H + h][D]  un-normalised output
-  float* logits;         // [l][b][h][Nv]    raw log2-domain logits of visual rows
+  float* logits;         // [l][b][h][Nv]    raw log2-domain logits of visual rows (this step's copy)
+  const float* logits_copy[2];  // both copies (a launch writes the one of its sequence parity)
+  float* head_stat;      // [l][b][h][2]     (max, 1/sum) of a pruning layer's merged softmax
   float* mass_by_id;     // [l][b][Nv]
   int* ids;              // [l][b][Nv]
   int* n_cur;            // [l][b]
@@ -83,6 +85,8 @@ struct StepParams {
   int t0_max;
   int static_rank;          // 1: keep the kept rows in top-index order, cut them without scoring
   const float* ext_scores;  // prefill with the caller's scores [layer_count][B][Nv]: selection only, no merge
+  int src_layer[kMaxLayers];  // the layer whose scores decide this layer's evictions (itself unless stage-shared)
+  int src_copy[kMaxLayers];   // which copy of the logits holds that layer's logits
 };
 
 // ------------------------------------------------------------------------------------------
@@ -374,7 +378,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
       T* gV = gK + (is_vis ? (long long)p.Nv * D : (long long)p.cap_txt * D);
       d.srcK = reinterpret_cast<const unsigned char*>(gK) + (size_t)r0 * ROWB;
       d.srcV = reinterpret_cast<const unsigned char*>(gV) + (size_t)r0 * ROWB;
-      d.want_logits = is_vis && p.ntgt[l_rel] < p.ncur[l_rel];
+      d.want_logits = is_vis && p.ntgt[l_rel] < p.ncur[l_rel] && p.src_layer[l_rel] == l;
       d.lb = (long long)l * p.B + b;
       d.wait_for = is_vis && d.lb != lb_ready ? p.req[l_rel] : 0;
       if (d.wait_for && ld_acquire(p.flags + d.lb) - d.wait_for >= 0) {  // looked up here, off the critical path
@@ -705,7 +709,11 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   }
   int* ids = p.ids + lb * Nv;
   float* mass_by_id = p.mass_by_id + lb * Nv;
-  const float* logits = p.logits + lb * H * Nv;
+  // the scores that decide come from this layer, or from its stage's pruning layer (same rows, same order)
+  const int src = p.src_layer[l_rel];
+  const long long lb_src = (long long)src * B + b;
+  const bool src_here = src >= p.layer_begin && src < p.layer_begin + p.layer_count;
+  const float* logits = p.logits_copy[p.src_copy[l_rel]] + lb_src * H * Nv;
   unsigned long long* s_key = reinterpret_cast<unsigned long long*>(smem);  // [Nv]
   int* s_hole = reinterpret_cast<int*>(smem + (size_t)Nv * 8);              // [Nv]
   int* s_mover = s_hole + Nv;                                               // [Nv]
@@ -728,10 +736,23 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
         pre[j] = h < H ? logits[(long long)h * Nv + ri] : -INFINITY;
       }
     }
-    for (int h = warp; h < H; h += kFinishWarps) {
-      float M, Lh;
-      merge_stats(ml, item0, nit, H, h, lane, M, Lh);
-      if (lane == 0) { s_M[h] = M; s_invL[h] = 1.f / Lh; }
+    if (src_here) {
+      const int ls = src - p.layer_begin;
+      const int nit_s = p.cvp[ls + 1] - p.cvp[ls] + p.ct;
+      const long long item0_s = (long long)p.lstart[ls] + (long long)b * nit_s;
+      for (int h = warp; h < H; h += kFinishWarps) {
+        float M, Lh;
+        merge_stats(ml, item0_s, nit_s, H, h, lane, M, Lh);
+        if (lane == 0) {
+          s_M[h] = M; s_invL[h] = 1.f / Lh;
+          if (src == l) { p.head_stat[2 * (lb * H + h)] = M; p.head_stat[2 * (lb * H + h) + 1] = 1.f / Lh; }
+        }
+      }
+    } else {  // the pruning layer ran in an earlier launch of this step: its statistics were kept
+      for (int h = tt; h < H; h += kFinishThreads) {
+        s_M[h] = p.head_stat[2 * (lb_src * H + h)];
+        s_invL[h] = p.head_stat[2 * (lb_src * H + h) + 1];
+      }
     }
   }
   __syncthreads();
@@ -980,7 +1001,7 @@ inline void make_fast_div(unsigned d, unsigned* mul, unsigned* shift) {
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 struct Layout {
-  size_t elem, cache, part_ml, part_acc, part_ml_bytes, part_acc_bytes, logits, mass, ids, n_cur, flags, text_len, status, stage_q, stage_k, stage_v,
+  size_t elem, cache, part_ml, part_acc, part_ml_bytes, part_acc_bytes, logits, logits_bytes, head_stat, mass, ids, n_cur, flags, text_len, status, stage_q, stage_k, stage_v,
       stage_o, total;
   long long lbh_stride;
   int cap_txt, chunk_rows, max_items;
@@ -1038,7 +1059,9 @@ Layout make_layout(const st3_config* c) {
   L.part_acc_bytes = align_up((size_t)L.max_items * c->num_heads * c->head_dim * sizeof(float), 256);
   L.part_ml = take(2 * L.part_ml_bytes);
   L.part_acc = take(2 * L.part_acc_bytes);
-  L.logits = take(lbh * (size_t)c->num_visual * sizeof(float));
+  L.logits_bytes = align_up(lbh * (size_t)c->num_visual * sizeof(float), 256);
+  L.logits = take(2 * L.logits_bytes);  // two copies, like the partials
+  L.head_stat = take(lbh * 2 * sizeof(float));
   L.mass = take(lb * (size_t)c->num_visual * sizeof(float));
   L.ids = take(lb * (size_t)c->num_visual * sizeof(int));
   L.n_cur = take(lb * sizeof(int));
@@ -1092,6 +1115,9 @@ struct st3_ctx {
   int seq;                     // sequence number of the next step's launches (starts at 1)
   unsigned counter_base;       // what the device work counter will read when the next launch starts
   std::vector<int> flag_req;   // per layer: sequence number of the last finish launch over it (0: none)
+  std::vector<int> logit_copy; // per layer: which copy holds the logits it wrote last
+  std::vector<int> logit_step; // per layer: the step those logits belong to (-1: none)
+  bool serialize_next;         // the next attention launch must wait for every earlier launch
 };
 
 namespace {
@@ -1136,7 +1162,7 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = (ctx->profiling || ingest) ? 0 : 1;
+    cfg.numAttrs = (ctx->profiling || ingest || ctx->serialize_next) ? 0 : 1;
     if (cudaLaunchKernelEx(&cfg, st3_attend_kernel<T, D>, p) != cudaSuccess) return ST3_ERR_CUDA;
   }
   if (e1) cudaEventRecord(e1, st);
@@ -1178,7 +1204,10 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
   p.flags = reinterpret_cast<int*>(ctx->ws + L.flags);
   p.seq = ctx->seq;
   p.counter_base = ctx->counter_base;
-  p.logits = reinterpret_cast<float*>(ctx->ws + L.logits);
+  p.logits = reinterpret_cast<float*>(ctx->ws + L.logits + (ctx->seq & 1) * L.logits_bytes);
+  p.logits_copy[0] = reinterpret_cast<const float*>(ctx->ws + L.logits);
+  p.logits_copy[1] = reinterpret_cast<const float*>(ctx->ws + L.logits + L.logits_bytes);
+  p.head_stat = reinterpret_cast<float*>(ctx->ws + L.head_stat);
   p.mass_by_id = reinterpret_cast<float*>(ctx->ws + L.mass);
   p.ids = reinterpret_cast<int*>(ctx->ws + L.ids);
   p.n_cur = reinterpret_cast<int*>(ctx->ws + L.n_cur);
@@ -1193,6 +1222,7 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
   p.k_in = prefill ? k : nullptr; p.v_in = prefill ? v : nullptr;
   p.t0_max = c.sys_len + c.num_visual + c.max_text_len;
   const int R = L.chunk_rows;
+  bool reads_older = false;  // this call's finish launch reads logits an earlier call wrote
   p.ct = ceil_div(c.sys_len + ctx->max_text + step, R);
   p.cvp[0] = 0;
   for (int i = 0; i < layer_count; ++i) {
@@ -1205,6 +1235,17 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
     if (c.static_rank && !prefill && tgt < ncur) ncur = tgt;  // cut first, then attend (Algorithm 3)
     p.ncur[i] = ncur;
     p.ntgt[i] = tgt < ncur ? tgt : ncur;
+    // whose scores decide: the layer's own, or (stage-shared) those of its stage's pruning layer
+    int src = l;
+    if (c.stage_shared && l >= c.first_prune_layer)
+      src = c.first_prune_layer + (l - c.first_prune_layer) / c.stride * c.stride;
+    p.src_layer[i] = src;
+    p.src_copy[i] = ctx->seq & 1;
+    if (src < layer_begin) {  // decided in an earlier call of this step
+      if (p.ntgt[i] < ncur && !ext_scores && ctx->logit_step[src] != step) return ST3_ERR_BAD_STATE;
+      p.src_copy[i] = ctx->logit_copy[src];
+      reads_older = true;
+    }
     const int cv = ceil_div(ncur, R);
     p.cvp[i + 1] = p.cvp[i] + cv;
     p.lstart[i] = c.batch * (p.cvp[i] + i * p.ct);
@@ -1235,7 +1276,14 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
     ctx->n_host[layer_begin + i] = p.ntgt[i];
     ctx->last_step[layer_begin + i] = step;
     ctx->flag_req[layer_begin + i] = ctx->seq;
+    if (p.src_layer[i] == layer_begin + i && p.ntgt[i] < p.ncur[i]) {  // it wrote logits in this launch
+      ctx->logit_copy[layer_begin + i] = ctx->seq & 1;
+      ctx->logit_step[layer_begin + i] = step;
+    }
   }
+  // Those logits are protected by no flag, so the launch that may overwrite them must not overlap this
+  // call's finish launch: it is launched without the programmatic attribute.
+  ctx->serialize_next = reads_older;
   ctx->seq++;
   ctx->counter_base += (unsigned)p.total_work;  // one fetch per work item (the first of each manager is fixed)
   ctx->last_stream = st;
@@ -1285,6 +1333,9 @@ st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, 
   ctx->seq = 1;
   ctx->counter_base = 0;
   ctx->flag_req.assign(cfg->num_layers, 0);
+  ctx->logit_copy.assign(cfg->num_layers, 0);
+  ctx->logit_step.assign(cfg->num_layers, -1);
+  ctx->serialize_next = false;
   ctx->profiling = false;
   ctx->ev_used = 0;
   ctx->attend_smem = kSlots * (2 * tile_bytes(cfg) + kQBytes);

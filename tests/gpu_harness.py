@@ -53,6 +53,8 @@ class GpuRun:
         self.out = torch.empty(self.ctx.io_shape(), dtype=self.ctx.dtype, device=self.dev)
         self.stats = {"exact": 0, "near-tie": 0, "units": 0}
         self.static = bool(cfg_overrides.get("static_rank", 0))
+        self.shared = bool(cfg_overrides.get("stage_shared", 0))
+        self._src_mass = {}          # (b, layer, step) -> oracle scores of a pruning layer
 
     def close(self):
         self.ctx.close()
@@ -126,6 +128,24 @@ class GpuRun:
         return {l: self.kept(l)[:2] for l in layers}
 
     # ------------------------------------------------------------------ checking
+    def stage_head(self, l):
+        wl = self.wl
+        if not self.shared or l < wl.first_prune_layer:
+            return l
+        return wl.first_prune_layer + (l - wl.first_prune_layer) // wl.stride * wl.stride
+
+    def _judge_follower(self, b, l, step, ids_before, n, where):
+        """A layer that follows its stage's pruning layer holds exactly the pruning layer's rows, in the
+        same order, and that set is judged against the pruning layer's oracle scores."""
+        src = self.stage_head(l)
+        ids, cnt, _ = self.kept(l)
+        ids_s, cnt_s, _ = self.kept(src)
+        assert int(cnt[b]) == int(cnt_s[b]) == n, where
+        assert np.array_equal(ids[b, :n], ids_s[b, :n]), f"{where}: rows differ from the pruning layer's"
+        verdict = check_kept(self._src_mass[(b, src, step)], np.asarray(ids_before), n, ids[b, :n])
+        self.stats[verdict] += 1
+        self.stats["units"] += 1
+
     def check_prefill_unit(self, b, l):
         wl, g, s = self.wl, self.g, self.sched
         t0 = wl.sys_len + wl.num_visual + int(g.text_len[b])
@@ -138,6 +158,10 @@ class GpuRun:
         ids, cnt, mass = self.kept(l)
         n = int(cnt[b])
         assert n == s.n0(l), (n, s.n0(l))
+        if self.stage_head(l) != l:
+            self._judge_follower(b, l, 0, np.arange(wl.num_visual), n, f"prefill b={b} l={l}")
+            return
+        self._src_mass[(b, l, 0)] = ref_mass
         self._judge(ref_mass, np.arange(wl.num_visual), s.n0(l), ids[b, :n], mass[b], trimmed=s.n0(l) < wl.num_visual,
                     where=f"prefill b={b} l={l}")
         if self.static and s.n0(l) < wl.num_visual:
@@ -166,6 +190,10 @@ class GpuRun:
         ids, cnt, mass = self.kept(l)
         n = int(cnt[b])
         assert n == s.n(l, step) == min(nb, s.n(l, step)), (n, s.n(l, step), nb)
+        if self.stage_head(l) != l:
+            self._judge_follower(b, l, step, ids_before, n, f"decode b={b} l={l} t={step}")
+            return
+        self._src_mass[(b, l, step)] = ref_mass
         self._judge(ref_mass, ids_before, n, ids[b, :n], mass[b], trimmed=n < nb, where=f"decode b={b} l={l} t={step}")
 
     def _judge(self, ref_mass, ids_before, k, got_ids, got_mass_by_id, trimmed, where):

@@ -125,3 +125,19 @@ def test_prefill_with_external_scores_then_decode(static_rank):
         assert run.ctx.status() == 0
     finally:
         run.close()
+
+
+@pytest.mark.parametrize("static_rank,lpc", [(0, None), (1, None), (0, 1), (0, 3)])
+def test_stage_shared_sets(static_rank, lpc):
+    """Layers between two pruning layers keep exactly the pruning layer's tokens (strided pruning)."""
+    wl = get_workload("tiny").scaled(dtype="bf16", head_dim=128, num_heads=4, num_layers=9, batch=2, sys_len=4,
+                                     num_visual=260, text_len_min=2, text_len_max=30, decode_steps=10,
+                                     first_prune_layer=2, stride=3, step_ratio_bp=1500, tau=10.0, num_planted=9)
+    stats = run_and_check(wl, 10, layers_per_call=lpc, stage_shared=1, static_rank=static_rank)
+    assert stats["units"] == 11 * 9 * 2
+
+
+def test_stage_shared_llava15_7b_first_steps():
+    wl = get_workload("llava15_7b")
+    stats = run_and_check(wl, 3, stage_shared=1)
+    assert stats["units"] == 32 * 4

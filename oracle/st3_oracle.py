@@ -296,6 +296,37 @@ def decode_step_static(cache: LayerCache, q, k_new, v_new, n_target: int):
     return out
 
 
+def attend_inherited(q_src, K_src, V_own):
+    """QK heredity (Eq. 6, Algorithm 2): a lazy layer reuses Softmax(Q^{l-n} (K^{l-n})^T / sqrt(d)) of the
+    last non-lazy layer and applies it to its OWN values.  q_src [H, D], K_src [H, T, D] are the source
+    layer's query and keys, V_own [H, T, D] the lazy layer's values, row j of both naming the same token."""
+    _, p = attend(q_src, K_src, np.zeros_like(np.asarray(V_own, dtype=np.float64)))
+    return np.matmul(p[:, None, :], np.asarray(V_own, dtype=np.float64))[:, 0, :]
+
+
+def decode_step_lazy(cache: LayerCache, cache_src: LayerCache, q_src, v_new, n_target: int, select_scores):
+    """One decode step of a lazy layer.  cache_src is the source layer's cache AFTER the source's own
+    append of this step and BEFORE its eviction; both caches must hold the same visual tokens in the
+    same order (they belong to one pruning stage).  The lazy layer appends only its value row, attends
+    with the inherited probabilities and then evicts what its stage's pruning layer evicts.
+    Returns out [H, D]."""
+    assert np.array_equal(cache.ids, cache_src.ids), "source and lazy layer must hold the same visual rows"
+    v_new = np.asarray(v_new, dtype=np.float64)
+    cache.V_txt = np.concatenate([cache.V_txt, v_new[:, None, :]], axis=1)
+    cache.K_txt = np.concatenate([cache.K_txt, np.zeros_like(v_new)[:, None, :]], axis=1)   # never read
+    K_src, _ = cache_src.rows()
+    _, V = cache.rows()
+    out = attend_inherited(q_src, K_src, V)
+    n_cur = cache.n_cur
+    n_new = min(n_cur, int(n_target))
+    if n_new < n_cur:
+        kept = select_top(np.asarray(select_scores, dtype=np.float64), cache.ids, n_new)
+        cache.K_vis = cache.K_vis[:, kept]
+        cache.V_vis = cache.V_vis[:, kept]
+        cache.ids = cache.ids[kept]
+    return out
+
+
 def boundary_scores(mass: np.ndarray, ids: np.ndarray, k: int):
     """(s_k, s_{k+1}): the k-th and (k+1)-th scores in selection order (None if absent)."""
     n = len(mass)

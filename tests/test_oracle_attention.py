@@ -82,3 +82,20 @@ def test_mass_accounts_for_all_probability():
     assert abs(m.sum() + non_visual - H) < 1e-12
     # transposed-operand guard: mass is a per-token sum over heads, not per-head sum over tokens
     assert np.allclose(m, np.array([sum(p[h, sys_len + i] for h in range(H)) for i in range(nv)]))
+
+
+def test_inherited_attention_is_the_sources_probabilities_on_own_values():
+    from oracle.st3_oracle import attend_inherited
+    r = np.random.default_rng(31)
+    H, T, D = 3, 14, 8
+    qs, Ks, Vs = r.standard_normal((H, D)), r.standard_normal((H, T, D)), r.standard_normal((H, T, D))
+    Vl = r.standard_normal((H, T, D))
+    _, p = attend(qs, Ks, Vs)
+    want = np.stack([sum(p[h, j] * Vl[h, j] for j in range(T)) for h in range(H)])
+    assert np.allclose(attend_inherited(qs, Ks, Vl), want, rtol=1e-13, atol=1e-15)
+    # with its own query, keys and values a layer "inherits" plain attention
+    assert np.allclose(attend_inherited(qs, Ks, Vs), attend(qs, Ks, Vs)[0], rtol=1e-13, atol=1e-15)
+    # library special case: SDPA with the source's q, k and the lazy layer's v
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(qs)[:, None, :], torch.from_numpy(Ks), torch.from_numpy(Vl))[:, 0, :]
+    assert np.allclose(attend_inherited(qs, Ks, Vl), ref.numpy(), rtol=1e-11, atol=1e-13)

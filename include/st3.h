@@ -84,6 +84,7 @@ typedef struct {
   int32_t static_rank;       /* 1: Algorithm 3 as printed, see below; 0: re-rank at every step   */
   int32_t stage_shared;      /* 1: the layers between two pruning layers keep the pruning layer's */
                              /*    choice (Sec. 3.2, strided pruning); 0: every layer chooses     */
+  uint64_t lazy_mask;        /* bit l set: layer l is lazy (QK heredity, Eq. 6, Algorithm 2)      */
   double tau;                /* Eq. 8: beta = cos(t*pi/(2 tau)) for t < tau, else 0             */
   double sigma;              /* only ST3_ANNEAL_EXP: beta = exp(-t/sigma)                       */
 } st3_config;
@@ -99,6 +100,14 @@ typedef struct {
  * exactly the tokens its pruning layer evicts (decided by the pruning layer's scores), so all layers
  * of a stage hold the same visual tokens in the same order.  Within one step the pruning layer must be
  * processed before (or in the same call as) the layers that follow it, else ST3_ERR_BAD_STATE. */
+
+/* lazy_mask: a lazy layer inherits Softmax(Q K^T / sqrt(d)) of the nearest lower layer that is not
+ * lazy and applies it to its own values (Eq. 6; Algorithm 2's A = U[-1]): its q and k_new inputs are
+ * ignored and its key rows are never read.  Source and lazy layer must hold the same tokens in the
+ * same order: both below first_prune_layer, or both in one pruning stage with stage_shared = 1 (else
+ * st3_create returns ST3_ERR_INVALID_ARG), and they must be processed in the same call (else
+ * ST3_ERR_UNSUPPORTED).  In this version a lazy layer re-reads its source's keys (same bytes as a
+ * normal layer); what it saves is the key cache and the key/query projections of the caller. */
 
 /* Scheduled visual-row count n(l, t) of layer `layer` after decode step `step` (0 = after
  * prefill).  Pure host function.  PVTP: layers below first_prune_layer keep everything; layer l

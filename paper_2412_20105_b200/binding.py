@@ -31,7 +31,7 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "num_layers", "num_heads", "head_dim", "dtype", "batch", "sys_len", "num_visual", "max_text_len",
         "max_decode_steps", "first_prune_layer", "stride", "first_ratio_bp", "step_ratio_bp", "anneal",
-        "disable_trim", "rows_per_chunk", "static_rank", "stage_shared")] + [("tau", C.c_double), ("sigma", C.c_double)]
+        "disable_trim", "rows_per_chunk", "static_rank", "stage_shared")] + [("lazy_mask", C.c_uint64), ("tau", C.c_double), ("sigma", C.c_double)]
 
 
 class St3Error(RuntimeError):
@@ -90,11 +90,11 @@ def _check(code: int, where: str):
 
 def make_config(*, num_layers, num_heads, head_dim, dtype, batch, sys_len, num_visual, max_text_len,
                 max_decode_steps, stride, step_ratio_bp, tau, first_prune_layer=3, first_ratio_bp=5000,
-                anneal=ST3_ANNEAL_COSINE, disable_trim=0, rows_per_chunk=0, sigma=20.0, static_rank=0, stage_shared=0) -> Config:
+                anneal=ST3_ANNEAL_COSINE, disable_trim=0, rows_per_chunk=0, sigma=20.0, static_rank=0, stage_shared=0, lazy_mask=0) -> Config:
     dt = {"f32": ST3_F32, "bf16": ST3_BF16}.get(dtype, dtype)
     return Config(num_layers, num_heads, head_dim, dt, batch, sys_len, num_visual, max_text_len,
                   max_decode_steps, first_prune_layer, stride, first_ratio_bp, step_ratio_bp, anneal,
-                  int(disable_trim), rows_per_chunk, int(static_rank), int(stage_shared), float(tau), float(sigma))
+                  int(disable_trim), rows_per_chunk, int(static_rank), int(stage_shared), int(lazy_mask), float(tau), float(sigma))
 
 
 def st3_schedule_count(cfg: Config, layer: int, step: int) -> int:

@@ -87,6 +87,7 @@ struct StepParams {
   const float* ext_scores;  // prefill with the caller's scores [layer_count][B][Nv]: selection only, no merge
   int src_layer[kMaxLayers];  // the layer whose scores decide this layer's evictions (itself unless stage-shared)
   int src_copy[kMaxLayers];   // which copy of the logits holds that layer's logits
+  int lazy_src[kMaxLayers];   // relative index of the layer whose q and K a lazy layer inherits (-1: its own)
 };
 
 // ------------------------------------------------------------------------------------------
@@ -330,8 +331,8 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
     // A decoded work item, held in registers until its slot is free.
     struct Dec {
       bool valid, has_new;
-      int nrows, nbulk, want_logits, wait_for;
-      long long slot, lbh, oidx, glog, lb;
+      int nrows, nbulk, want_logits, wait_for, wait_for_k;
+      long long slot, lbh, oidx, oidx_q, glog, lb, lb_k;
       const unsigned char *srcK, *srcV;
       T *newK, *newV;
       uint4 nv[NV];
@@ -373,9 +374,15 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
       d.nbulk = nrows - (d.has_new ? 1 : 0);
       d.lbh = ((long long)l * p.B + b) * H + h;
       d.oidx = ((long long)l_rel * p.B + b) * H + h;
+      // QK heredity (Eq. 6): a lazy layer attends with the query and the keys of its source layer and
+      // its own values; the two layers hold the same tokens in the same order
+      const int ls = p.lazy_src[l_rel];
+      d.oidx_q = ls < 0 ? d.oidx : ((long long)ls * p.B + b) * H + h;
+      const long long lbh_k = ls < 0 ? d.lbh : ((long long)(p.layer_begin + ls) * p.B + b) * H + h;
       T* blk = reinterpret_cast<T*>(p.cache) + d.lbh * p.lbh_stride;
-      T* gK = is_vis ? blk : blk + 2LL * p.Nv * D;
-      T* gV = gK + (is_vis ? (long long)p.Nv * D : (long long)p.cap_txt * D);
+      T* blk_k = reinterpret_cast<T*>(p.cache) + lbh_k * p.lbh_stride;
+      T* gK = is_vis ? blk_k : blk_k + 2LL * p.Nv * D;
+      T* gV = is_vis ? blk + (long long)p.Nv * D : blk + 2LL * p.Nv * D + (long long)p.cap_txt * D;
       d.srcK = reinterpret_cast<const unsigned char*>(gK) + (size_t)r0 * ROWB;
       d.srcV = reinterpret_cast<const unsigned char*>(gV) + (size_t)r0 * ROWB;
       d.want_logits = is_vis && p.ntgt[l_rel] < p.ncur[l_rel] && p.src_layer[l_rel] == l;
@@ -385,14 +392,17 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
         d.wait_for = 0;
         lb_ready = d.lb;
       }
+      d.lb_k = (long long)(ls < 0 ? l : p.layer_begin + ls) * p.B + b;
+      d.wait_for_k = is_vis && ls >= 0 ? p.req[ls] : 0;  // the source's rows as well
       d.glog = d.lbh * p.Nv + r0;
       d.slot = (long long)item * H + h;
       if (d.has_new) {
         // newest row: fetched from the step's inputs now, stored when the slot is free
-        d.newK = gK + (long long)(seg_rows - 1) * D;
+        d.newK = ls < 0 ? gK + (long long)(seg_rows - 1) * D : nullptr;  // the source layer stores its own key
         d.newV = gV + (long long)(seg_rows - 1) * D;
         if (lane < 2 * LN) {
-          const T* src = reinterpret_cast<const T*>(lane / LN ? p.v_new : p.k_new) + d.oidx * D;
+          const T* src = lane / LN ? reinterpret_cast<const T*>(p.v_new) + d.oidx * D
+                                   : reinterpret_cast<const T*>(p.k_new) + d.oidx_q * D;
 #pragma unroll
           for (int i = 0; i < NV; ++i) d.nv[i] = __ldg(reinterpret_cast<const uint4*>(src) + (lane % LN) + i * LN);
         }
@@ -404,13 +414,15 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
         if (!flag_wait(p.flags + d.lb, d.wait_for, abort_flag, p.status)) return;
         lb_ready = d.lb;
       }
+      if (d.wait_for_k && !flag_wait(p.flags + d.lb_k, d.wait_for_k, abort_flag, p.status)) return;
       if (d.has_new) {
         if (lane < 2 * LN) {
           const int kv = lane / LN;
 #pragma unroll
           for (int i = 0; i < NV; ++i) {
             const int cc = (lane % LN) + i * LN;
-            reinterpret_cast<uint4*>(kv ? d.newV : d.newK)[cc] = d.nv[i];
+            T* dstg = kv ? d.newV : d.newK;
+            if (dstg) reinterpret_cast<uint4*>(dstg)[cc] = d.nv[i];
             *reinterpret_cast<uint4*>((kv ? sV : sK) + (size_t)(d.nrows - 1) * ROWB + cc * 16) = d.nv[i];
           }
         }
@@ -421,7 +433,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
         sd.nrows = d.nrows; sd.want_logits = d.want_logits; sd.glog = d.glog;
         const uint32_t kb = (uint32_t)d.nbulk * ROWB;
         mbar_expect_tx(&s_fullK[s][g], kb + ROWB);  // K rows + the query (D elements = ROWB bytes)
-        bulk_g2s(sQ, reinterpret_cast<const T*>(p.q) + d.oidx * D, ROWB, &s_fullK[s][g]);
+        bulk_g2s(sQ, reinterpret_cast<const T*>(p.q) + d.oidx_q * D, ROWB, &s_fullK[s][g]);
         if (kb) {
           bulk_g2s(sK, d.srcK, kb, &s_fullK[s][g]);
           mbar_expect_tx(&s_fullV[s][g], kb);
@@ -1023,6 +1035,19 @@ bool valid_config(const st3_config* c) {
   if ((c->anneal == ST3_ANNEAL_COSINE || c->anneal == ST3_ANNEAL_LINEAR) && !(c->tau > 0.0)) return false;
   if (c->anneal == ST3_ANNEAL_EXP && !(c->sigma > 0.0)) return false;
   if (c->rows_per_chunk < 0 || c->rows_per_chunk > kMaxChunkRows) return false;
+  // lazy layers (QK heredity): the source is the nearest lower layer that is not lazy, and it must hold
+  // the same tokens in the same order, i.e. sit in the same pruning stage with stage_shared set
+  for (int l = 0; l < c->num_layers; ++l) {
+    if (!(c->lazy_mask >> l & 1ull)) continue;
+    if (l == 0) return false;
+    int sl = l - 1;
+    while (sl > 0 && (c->lazy_mask >> sl & 1ull)) --sl;
+    if (c->lazy_mask >> sl & 1ull) return false;
+    if (c->disable_trim || l < c->first_prune_layer) continue;
+    if (!c->stage_shared || sl < c->first_prune_layer) return false;
+    if ((l - c->first_prune_layer) / c->stride != (sl - c->first_prune_layer) / c->stride) return false;
+  }
+  if (c->num_layers < 64 && (c->lazy_mask >> c->num_layers)) return false;
   return true;
 }
 
@@ -1235,6 +1260,13 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
     if (c.static_rank && !prefill && tgt < ncur) ncur = tgt;  // cut first, then attend (Algorithm 3)
     p.ncur[i] = ncur;
     p.ntgt[i] = tgt < ncur ? tgt : ncur;
+    p.lazy_src[i] = -1;
+    if (c.lazy_mask >> l & 1ull) {
+      int sl = l - 1;
+      while (sl > 0 && (c.lazy_mask >> sl & 1ull)) --sl;
+      if (sl < layer_begin) return ST3_ERR_UNSUPPORTED;  // a lazy layer and its source must share a call
+      p.lazy_src[i] = sl - layer_begin;
+    }
     // whose scores decide: the layer's own, or (stage-shared) those of its stage's pruning layer
     int src = l;
     if (c.stage_shared && l >= c.first_prune_layer)

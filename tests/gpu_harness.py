@@ -55,6 +55,7 @@ class GpuRun:
         self.static = bool(cfg_overrides.get("static_rank", 0))
         self.shared = bool(cfg_overrides.get("stage_shared", 0))
         self._src_mass = {}          # (b, layer, step) -> oracle scores of a pruning layer
+        self.lazy_mask = int(cfg_overrides.get("lazy_mask", 0))
 
     def close(self):
         self.ctx.close()
@@ -125,9 +126,24 @@ class GpuRun:
 
     def snapshot(self, layers):
         """{layer: (ids [B, Nv], count [B])} of the current device state."""
-        return {l: self.kept(l)[:2] for l in layers}
+        snap = {l: self.kept(l)[:2] for l in layers}
+        for l in list(snap):
+            src = self.lazy_source(l)
+            if src is not None and src not in snap:
+                snap[src] = self.kept(src)[:2]
+        self._before_all = snap
+        return snap
 
     # ------------------------------------------------------------------ checking
+    def lazy_source(self, l):
+        """The layer whose q and K layer l inherits (QK heredity), or None."""
+        if not (self.lazy_mask >> l) & 1:
+            return None
+        s = l - 1
+        while (self.lazy_mask >> s) & 1:
+            s -= 1
+        return s
+
     def stage_head(self, l):
         wl = self.wl
         if not self.shared or l < wl.first_prune_layer:
@@ -153,6 +169,11 @@ class GpuRun:
         q = g.queries([0], [l])[0, 0, b]
         ref_out, ref_mass, _ = O.prefill_select(f64(q), f64(K[0, 0]), f64(V[0, 0]), wl.sys_len, wl.num_visual,
                                                 s.n0(l))
+        src = self.lazy_source(l)
+        if src is not None:     # inherited probabilities: the source's query and keys, this layer's values
+            Ks, _ = g.kv_rows([b], [src], range(t0))
+            qs = g.queries([0], [src])[0, 0, b]
+            ref_out = O.attend_inherited(f64(qs), f64(Ks[0, 0]), f64(V[0, 0]))
         got = f64(self.out[l, b])
         assert_out_close(got, ref_out, wl.dtype, f"prefill out b={b} l={l}")
         ids, cnt, mass = self.kept(l)
@@ -173,6 +194,33 @@ class GpuRun:
         ids_b, cnt_b = before
         nb = int(cnt_b[b])
         cache = rebuild_cache(wl, g, b, l, ids_b[b, :nb], step - 1)
+        src = self.lazy_source(l)
+        if src is not None:
+            assert not self.static
+            ids_s, cnt_s = self._before_all[src]
+            assert int(cnt_s[b]) == nb and np.array_equal(ids_s[b, :nb], ids_b[b, :nb])
+            cache_src = rebuild_cache(wl, g, b, src, ids_s[b, :nb], step - 1)
+            kn_s = f64(self.kn_cur[src, b])
+            cache_src.K_txt = np.concatenate([cache_src.K_txt, kn_s[:, None, :]], axis=1)
+            cache_src.V_txt = np.concatenate([cache_src.V_txt, np.zeros_like(kn_s)[:, None, :]], axis=1)
+            head = self.stage_head(l)
+            sel = self._src_mass.get((b, head, step)) if head != l else None
+            n_t = s.n(l, step)
+            if sel is None:
+                assert n_t >= nb, "a lazy layer that evicts must follow a pruning layer"
+                sel = np.zeros(nb)
+            ref_out = O.decode_step_lazy(cache, cache_src, f64(self.q_cur[src, b]), f64(self.vn_cur[l, b]), n_t, sel)
+            assert_out_close(f64(self.out[l, b]), ref_out, wl.dtype, f"lazy decode out b={b} l={l} t={step}")
+            ids, cnt, _ = self.kept(l)
+            n = int(cnt[b])
+            assert n == min(nb, n_t)
+            if head != l:
+                self._judge_follower(b, l, step, ids_b[b, :nb], n, f"lazy decode b={b} l={l} t={step}")
+            else:
+                assert np.array_equal(ids[b, :n], ids_b[b, :n])
+                self.stats["exact"] += 1
+                self.stats["units"] += 1
+            return
         if self.static:
             ref_out = O.decode_step_static(cache, f64(self.q_cur[l, b]), f64(self.kn_cur[l, b]), f64(self.vn_cur[l, b]),
                                            s.n(l, step))
@@ -219,7 +267,9 @@ class GpuRun:
         toks = list(range(wl.sys_len)) + list(range(wl.sys_len + wl.num_visual, wl.sys_len + wl.num_visual + text)) \
             + [g.gen_token(s) for s in range(1, step + 1)]
         Kt, Vt = g.kv_rows([b], [l], toks)
-        assert torch.equal(kt[:len(toks)].cpu(), Kt[0, 0, h]) and torch.equal(vt[:len(toks)].cpu(), Vt[0, 0, h])
+        assert torch.equal(vt[:len(toks)].cpu(), Vt[0, 0, h])
+        nk = len(toks) - step if self.lazy_source(l) is not None else len(toks)   # a lazy layer stores no new keys
+        assert torch.equal(kt[:nk].cpu(), Kt[0, 0, h, :nk])
 
 
 def run_and_check(wl: Workload, steps, check_steps=None, units=None, layers_per_call=None, rows_checks=2, **cfg):

@@ -37,7 +37,7 @@ def test_every_declared_symbol_is_exported():
 def test_config_struct_matches_header_order():
     hdr = open(os.path.join(ROOT, "include", "st3.h")).read()
     body = re.search(r"typedef struct \{(.*?)\} st3_config;", hdr, re.S).group(1)
-    fields = re.findall(r"(?:int32_t|double)\s+([a-z_]+);", body)
+    fields = re.findall(r"(?:int32_t|uint64_t|double)\s+([a-z_]+);", body)
     assert fields == [f[0] for f in B.Config._fields_]
 
 

@@ -141,3 +141,24 @@ def test_stage_shared_llava15_7b_first_steps():
     wl = get_workload("llava15_7b")
     stats = run_and_check(wl, 3, stage_shared=1)
     assert stats["units"] == 32 * 4
+
+
+def test_qk_heredity_lazy_layers():
+    """Lazy layers attend with their source layer's probabilities and their own values (Eq. 6)."""
+    wl = get_workload("tiny").scaled(dtype="bf16", head_dim=128, num_heads=4, num_layers=9, batch=2, sys_len=4,
+                                     num_visual=260, text_len_min=2, text_len_max=30, decode_steps=10,
+                                     first_prune_layer=2, stride=3, step_ratio_bp=1500, tau=10.0, num_planted=9)
+    # stages: [2,3,4] [5,6,7] [8]; lazy: 1 (source 0, unpruned), 3 and 4 (source 2), 7 (source 6)
+    lazy = (1 << 1) | (1 << 3) | (1 << 4) | (1 << 7)
+    stats = run_and_check(wl, 10, stage_shared=1, lazy_mask=lazy)
+    assert stats["units"] == 11 * 9 * 2
+
+
+def test_qk_heredity_configuration_errors():
+    from paper_2412_20105_b200 import binding as B
+    wl = get_workload("tiny").scaled(num_layers=9, first_prune_layer=2, stride=3, step_ratio_bp=1500)
+    for kw in (dict(lazy_mask=1), dict(lazy_mask=1 << 3), dict(lazy_mask=1 << 5, stage_shared=1),
+               dict(lazy_mask=1 << 2, stage_shared=1), dict(lazy_mask=1 << 9, stage_shared=1)):
+        with pytest.raises(B.St3Error):
+            B.st3_workspace_size(B.config_from_workload(wl, **kw))
+    B.st3_workspace_size(B.config_from_workload(wl, lazy_mask=(1 << 3) | (1 << 4), stage_shared=1))

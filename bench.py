@@ -37,19 +37,22 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of the attention kernel measured once with ncu (dram__bytes_read.sum +
 # dram__bytes_write.sum over three launches of the llava15_7b workload, see profiles/), as a
 # ratio to the algorithmic bytes of the same launches.  Valid only for the kernel source it was
-# taken on: the hash covers the attention kernel's section of csrc/st3.cu.
+# taken on: the hash covers csrc/st3_common.cuh and csrc/st3_attend.cuh.
 ATTEND_TRAFFIC = {"workload": "llava15_7b", "ratio": 1.026,
                   "kernel_sha256": "b172c5ec0faf526fdabff4b01223ee0824c8475ce42057bb56d4b469509315f9"}
 
 
-def attend_traffic_ratio(workload_name):
+def attend_kernel_sha256():
     import hashlib
+    h = hashlib.sha256()
+    for f in ("st3_common.cuh", "st3_attend.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2412_20105_b200", "csrc", f), "rb").read())
+    return h.hexdigest()
+
+
+def attend_traffic_ratio(workload_name):
     try:
-        src = open(os.path.join(ROOT, "paper_2412_20105_b200", "csrc", "st3.cu")).read()
-        a = src.index("// Attention (Eq. 2, last row) + raw visual logits + KV append")
-        b = src.index("// Merge partials, visual scores")
-        if hashlib.sha256(src[a:b].encode()).hexdigest() == ATTEND_TRAFFIC["kernel_sha256"] \
-                and workload_name == ATTEND_TRAFFIC["workload"]:
+        if attend_kernel_sha256() == ATTEND_TRAFFIC["kernel_sha256"] and workload_name == ATTEND_TRAFFIC["workload"]:
             return ATTEND_TRAFFIC["ratio"]
     except Exception:
         pass

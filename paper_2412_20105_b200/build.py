@@ -8,7 +8,8 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 LIB = os.path.join(PKG, "libst3.so")
 SOURCES = [os.path.join(PKG, "csrc", "st3.cu")]
-HEADERS = [os.path.join(ROOT, "include", "st3.h")]
+HEADERS = [os.path.join(ROOT, "include", "st3.h")] + [
+    os.path.join(PKG, "csrc", f) for f in ("st3_common.cuh", "st3_attend.cuh", "st3_finish.cuh")]
 
 
 def needs_build() -> bool:
@@ -23,7 +24,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-o", LIB] + SOURCES
+           "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", os.path.join(PKG, "csrc"), "-o", LIB] + SOURCES
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     subprocess.run(cmd, check=True)

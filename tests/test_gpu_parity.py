@@ -162,3 +162,24 @@ def test_qk_heredity_configuration_errors():
         with pytest.raises(B.St3Error):
             B.st3_workspace_size(B.config_from_workload(wl, **kw))
     B.st3_workspace_size(B.config_from_workload(wl, lazy_mask=(1 << 3) | (1 << 4), stage_shared=1))
+
+
+def test_paper_style_configuration_on_llava15_7b():
+    """7B schedule with shared stages and the paper's lazy pattern inside the last full stage
+    (layers 29 and 30 inherit layer 28; layer 31 starts a new stage and cannot be lazy)."""
+    wl = get_workload("llava15_7b")
+    lazy = (1 << 29) | (1 << 30)
+    steps = [0, 1, 2, 60, 255, 256]
+    stats = run_and_check(wl, wl.decode_steps, check_steps=steps, stage_shared=1, lazy_mask=lazy)
+    assert stats["units"] == 32 * len(steps)
+
+
+def test_stage_shared_13b_sampled():
+    wl = get_workload("llava15_13b_b16")
+    units = _sampled_units(wl, 6, 11) + [(0, 3), (0, 4), (0, 6), (5, 7), (5, 8)]
+    units = sorted(set(units), key=lambda u: (u[1], u[0]))
+    # a follower is judged against its pruning layer: make sure every sampled follower has it in the list
+    heads = sorted(set((b, 3 + (l - 3) // 4 * 4) for b, l in units if l >= 3))
+    units = sorted(set(units) | set(heads), key=lambda u: (u[1], u[0]))
+    stats = run_and_check(wl, 40, check_steps=[0, 1, 20, 40], units=units, rows_checks=1, stage_shared=1)
+    assert stats["units"] == len(units) * 4

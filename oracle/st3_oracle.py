@@ -128,6 +128,22 @@ def attend(q: np.ndarray, K: np.ndarray, V: np.ndarray):
     return out, p
 
 
+def causal_attention(Q: np.ndarray, K: np.ndarray, V: np.ndarray):
+    """Eq. 2 in full: A = Softmax((Q K^T + M) / sqrt(d)), out = A V, with M masking the strict upper
+    triangle (row i sees keys 0..i).  Q, K, V [H, T, D].  Returns (out [H, T, D], A [H, T, T])."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    T, d = Q.shape[1], Q.shape[2]
+    logits = np.matmul(Q, np.swapaxes(K, 1, 2)) / math.sqrt(d)            # [H, T, T]
+    mask = np.triu(np.ones((T, T), dtype=bool), k=1)
+    logits = np.where(mask[None], -np.inf, logits)
+    logits = logits - logits.max(axis=2, keepdims=True)
+    e = np.exp(logits)
+    A = e / e.sum(axis=2, keepdims=True)
+    return np.matmul(A, V), A
+
+
 def visual_mass(p: np.ndarray, vis_begin: int, n_vis: int) -> np.ndarray:
     """alpha: the query's attention on each visual token, summed over heads."""
     return p[:, vis_begin:vis_begin + n_vis].sum(axis=0)

@@ -1,4 +1,6 @@
 """Pins for the oracle's attention and score arithmetic (Eq. 2, last row)."""
+import math
+
 import numpy as np
 import torch
 
@@ -99,3 +101,22 @@ def test_inherited_attention_is_the_sources_probabilities_on_own_values():
     ref = torch.nn.functional.scaled_dot_product_attention(
         torch.from_numpy(qs)[:, None, :], torch.from_numpy(Ks), torch.from_numpy(Vl))[:, 0, :]
     assert np.allclose(attend_inherited(qs, Ks, Vl), ref.numpy(), rtol=1e-11, atol=1e-13)
+
+
+def test_causal_attention_against_sdpa_and_its_last_row_against_attend():
+    from oracle.st3_oracle import causal_attention
+    r = np.random.default_rng(41)
+    H, T, D = 2, 19, 8
+    Q, K, V = r.standard_normal((H, T, D)), r.standard_normal((H, T, D)), r.standard_normal((H, T, D))
+    out, A = causal_attention(Q, K, V)
+    ref = torch.nn.functional.scaled_dot_product_attention(torch.from_numpy(Q), torch.from_numpy(K),
+                                                           torch.from_numpy(V), is_causal=True)
+    assert np.allclose(out, ref.numpy(), rtol=1e-11, atol=1e-13)
+    assert np.allclose(A.sum(axis=2), 1.0) and np.all(np.triu(A, k=1) == 0)      # rows sum to 1, no look-ahead
+    assert np.allclose(out[:, 0], V[:, 0])                                       # the first token sees itself only
+    o_last, p_last = attend(Q[:, -1], K, V)                                      # the decode row of Eq. 2
+    assert np.allclose(out[:, -1], o_last, rtol=1e-12, atol=1e-14) and np.allclose(A[:, -1], p_last, rtol=1e-12)
+    # brute force of one entry
+    i, h = 7, 1
+    w = np.array([math.exp(float(Q[h, i] @ K[h, j]) / math.sqrt(D)) for j in range(i + 1)])
+    assert np.allclose(out[h, i], (w[:, None] * V[h, :i + 1]).sum(axis=0) / w.sum(), rtol=1e-12)

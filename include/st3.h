@@ -199,6 +199,23 @@ st3_status st3_profile_read(st3_ctx* ctx, double* attn_ms, double* finish_ms, in
 /* Total kernels this context has launched so far (host counter). */
 int64_t st3_launch_count(const st3_ctx* ctx);
 
+/* Causal self-attention of a whole prompt (Eq. 2: A = Softmax((Q K^T + M)/sqrt(d)), out = A V, row i sees
+ * keys 0..i), the step that produces what st3_prefill_select consumes.  Runs on the tcgen05 tensor cores;
+ * bf16 and head_dim 128 only (else ST3_ERR_UNSUPPORTED).  A "head instance" is one (sequence, head) pair.
+ *   q, k, v     dev [num_inst][seq_len][128] bf16, instance = sequence * num_heads + head
+ *   out         dev [num_inst][seq_len][128] bf16
+ *   head_probs  dev [num_inst][num_visual] fp32 scratch (the last row's probabilities per head)
+ *   scores      dev [num_inst / num_heads][num_visual] fp32: the last query row's attention on the visual
+ *               positions [sys_len, sys_len + num_visual), summed over heads -- the alpha of Sec. 3.2 that
+ *               Eq. 3 uses to prune the NEXT layer (feed it to st3_prefill_select_scored).
+ *               head_probs and scores may be NULL when num_visual is 0.
+ *   dev_status  dev int, may be NULL: ST3_DEV_COPY_TIMEOUT is OR-ed in if a copy or an MMA never completes
+ * Needs no context and no workspace beyond head_probs. */
+st3_status st3_prefill_attend(const void* q, const void* k, const void* v, void* out, float* head_probs,
+                              float* scores, int* dev_status, int32_t num_inst, int32_t num_heads,
+                              int32_t seq_len, int32_t head_dim, int32_t dtype, int32_t sys_len,
+                              int32_t num_visual, void* cuda_stream);
+
 /* Attention of one query per head over dense K/V with NO workspace and no allocation of any kind
  * (the paper has no counterpart; this exists for callers that may not allocate device memory:
  * a plugin handed only its input and output tensors, code running inside a region whose memory

@@ -23,7 +23,7 @@ EXPORTS = ["st3_schedule_count", "st3_workspace_size", "st3_create", "st3_prefil
            "st3_prefill_select_scored", "st3_decode_step",
            "st3_decode_step_host", "st3_get_kept", "st3_get_rows", "st3_get_status", "st3_rows_held",
            "st3_profile_enable", "st3_profile_read", "st3_launch_count", "st3_status_string", "st3_destroy",
-           "st3_attend_noalloc"]
+           "st3_attend_noalloc", "st3_prefill_attend"]
 
 
 class Config(C.Structure):
@@ -76,6 +76,7 @@ def load():
     lib.st3_status_string.restype = C.c_char_p
     lib.st3_destroy.argtypes = [vp]
     lib.st3_attend_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.st3_prefill_attend.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp]
     for name in EXPORTS:
         if name not in ("st3_schedule_count", "st3_launch_count", "st3_status_string"):
             getattr(lib, name).restype = C.c_int
@@ -181,6 +182,14 @@ def st3_status_string(code: int) -> str:
 
 def st3_destroy(ctx):
     _check(load().st3_destroy(ctx), "st3_destroy")
+
+
+def st3_prefill_attend(q, k, v, out, head_probs, scores, dev_status, num_inst, num_heads, seq_len, head_dim, dtype,
+                       sys_len, num_visual, stream=0):
+    """Causal attention of a whole prompt on the tensor cores (device addresses; see st3.h)."""
+    dt = {"f32": ST3_F32, "bf16": ST3_BF16}.get(dtype, dtype)
+    _check(load().st3_prefill_attend(q, k, v, out, head_probs, scores, dev_status, num_inst, num_heads, seq_len,
+                                     head_dim, dt, sys_len, num_visual, stream), "st3_prefill_attend")
 
 
 def st3_attend_noalloc(q, k, v, out, num_heads, num_rows, head_dim, dtype, stream=0):

@@ -7,7 +7,7 @@ import subprocess
 PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 LIB = os.path.join(PKG, "libst3.so")
-SOURCES = [os.path.join(PKG, "csrc", "st3.cu")]
+SOURCES = [os.path.join(PKG, "csrc", "st3.cu"), os.path.join(PKG, "csrc", "st3_prefill.cu")]
 HEADERS = [os.path.join(ROOT, "include", "st3.h")] + [
     os.path.join(PKG, "csrc", f) for f in ("st3_common.cuh", "st3_attend.cuh", "st3_finish.cuh")]
 

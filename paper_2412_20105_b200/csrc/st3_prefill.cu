@@ -1,0 +1,358 @@
+// Causal prompt attention (Eq. 2 in full) on the 5th-generation tensor cores: tcgen05.mma with
+// accumulators in tensor memory, operands staged in shared memory by TMA, for bf16 and D = 128.
+//
+// One block per (head instance, 128-query tile).  Warp 4 is the control warp: it issues the TMA loads
+// and the MMAs.  Warps 0-3 own one query row per thread (thread i <-> TMEM lane i), so the softmax needs
+// no cross-thread reduction.  Two passes over the key tiles 0..q_tile:
+//   pass 1   S = Q K^T (tcgen05.mma, 128x128x128), rows keep a running max and sum;
+//   pass 2   S again, P = exp2(S - max) / sum as bf16 into shared memory, O += P V (second MMA).
+// Recomputing S costs half again the tensor work but needs no rescaling of O in tensor memory.
+// The last query row's probabilities on the visual positions are written per head and summed over
+// heads by a second small kernel: the scores alpha (Sec. 3.2) that prune the NEXT layer.
+//
+// Shared-memory operand layout: 128-byte swizzle, K-major tiles of [rows][64 bf16] (what a TMA box with
+// CU_TENSOR_MAP_SWIZZLE_128B writes); V is consumed as an MN-major B operand straight from the same
+// kind of box.  Every wait is bounded; a timeout sets the error word and lets the block finish.
+#include "st3_common.cuh"
+
+#include <cuda.h>
+
+namespace {
+
+constexpr int kPfThreads = 160;       // 4 softmax warps + the control warp
+constexpr int kTile = 128;            // queries and keys per tile
+constexpr int kPfD = 128;
+constexpr int kBoxBytes = 128 * 128;  // one TMA box: 128 rows x 64 bf16
+constexpr int kTileBytes2 = 2 * kBoxBytes;
+constexpr uint32_t kTmemCols = 256;   // S in columns [0,128), O in [128,256)
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst)),
+      "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cta(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Bounded wait; false after ~2 s (the caller sets the error word and stops issuing work).
+__device__ __forceinline__ bool pf_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > kWaitCycles) return false;
+  }
+  return true;
+}
+// Shared-memory matrix descriptor: 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
+  return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      :
+      : "r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 128.
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescS = kIdescBase;               // A and B K-major
+constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);  // B (= V) MN-major
+
+struct PrefillParams {
+  __nv_bfloat16* out;   // [num_inst][T][128]
+  float* head_probs;    // [num_inst][num_visual] last-row probabilities per head
+  int* status;          // error word (may be null)
+  int T, sys_len, num_visual;
+};
+
+__global__ void __launch_bounds__(kPfThreads, 1)
+st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                          const __grid_constant__ CUtensorMap map_v, const PrefillParams p) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  // the dynamic window is only 16-byte aligned by contract: round up to the 1024 bytes the swizzle needs
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* sQ = smem;
+  unsigned char* sK = sQ + kTileBytes2;
+  unsigned char* sV = sK + kTileBytes2;
+  unsigned char* sP = sV + kTileBytes2;
+  __shared__ __align__(8) uint64_t bar_q, bar_kv, bar_s, bar_read, bar_o;
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_fail;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int qt = blockIdx.x, inst = blockIdx.y;
+  const int T = p.T;
+  const int row_base = inst * T;  // first row of this instance in the [num_inst * T][128] tensors
+  const int nkt = qt + 1;         // causal: key tiles 0..qt
+
+  if (tid == 0) {
+    mbar_init(&bar_q, 1); mbar_init(&bar_kv, 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
+    mbar_init(&bar_read, 128);
+    s_fail = 0;
+    mbar_fence_init();
+  }
+  __syncthreads();
+  if (warp == 4) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem)), "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = s_tmem;
+  const uint32_t tmem_S = tmem, tmem_O = tmem + 128;
+  volatile int* fail = &s_fail;
+
+  if (warp == 4) {
+    // ===================== control warp =====================
+    uint32_t ph_kv = 0, ph_s = 0, ph_read = 0, ph_o = 0;
+    bool ok = true;
+    if (lane == 0) {
+      mbar_expect_tx(&bar_q, kTileBytes2);
+      tma_load_2d(sQ, &map_q, 0, row_base + qt * kTile, &bar_q);
+      tma_load_2d(sQ + kBoxBytes, &map_q, 64, row_base + qt * kTile, &bar_q);
+    }
+    ok = pf_wait(&bar_q, 0);
+    for (int pass = 0; pass < 2 && ok; ++pass) {
+      for (int kt = 0; kt < nkt && ok; ++kt) {
+        if (lane == 0) {
+          mbar_expect_tx(&bar_kv, pass ? 2 * kTileBytes2 : kTileBytes2);
+          tma_load_2d(sK, &map_k, 0, row_base + kt * kTile, &bar_kv);
+          tma_load_2d(sK + kBoxBytes, &map_k, 64, row_base + kt * kTile, &bar_kv);
+          if (pass) {
+            tma_load_2d(sV, &map_v, 0, row_base + kt * kTile, &bar_kv);
+            tma_load_2d(sV + kBoxBytes, &map_v, 64, row_base + kt * kTile, &bar_kv);
+          }
+        }
+        ok = pf_wait(&bar_kv, ph_kv); ph_kv ^= 1;
+        if (!ok) break;
+        tc_fence_after();
+        if (lane == 0) {
+          // S = Q K^T: 8 steps of 16 along the head dimension
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks) {
+            const uint32_t off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
+            umma_bf16(tmem_S, smem_desc(smem_u32(sQ) + off, 16), smem_desc(smem_u32(sK) + off, 16), kIdescS, ks > 0);
+          }
+          umma_commit(&bar_s);
+        }
+        __syncwarp();
+        // the softmax warps have read S (pass 1) or have written P (pass 2)
+        ok = pf_wait(&bar_read, ph_read); ph_read ^= 1;
+        if (!ok) break;
+        if (pass) {
+          tc_fence_after();
+          if (lane == 0) {
+            // O += P V: 8 steps of 16 keys; V is the MN-major operand (two 64-dim boxes 16 KB apart)
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+              const uint32_t offp = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
+              umma_bf16(tmem_O, smem_desc(smem_u32(sP) + offp, 16), smem_desc(smem_u32(sV) + ks * 2048, kBoxBytes),
+                        kIdescPV, (kt > 0 || ks > 0));
+            }
+            umma_commit(&bar_o);
+          }
+          __syncwarp();
+          ok = pf_wait(&bar_o, ph_o); ph_o ^= 1;   // K, V and P tiles are free again (and, at the end, O is complete)
+        } else {
+          ok = pf_wait(&bar_s, ph_s);              // the MMA is done with the K tile
+        }
+        ph_s ^= 1;
+      }
+    }
+    if (!ok) { *fail = 1; if (lane == 0 && p.status) atomicOr(p.status, ST3_DEV_COPY_TIMEOUT); }
+  } else {
+    // ===================== softmax warps: thread <-> query row =====================
+    const int r = tid;                        // row inside the tile == TMEM lane
+    const int qi = qt * kTile + r;            // query position inside the instance
+    const bool live = qi < T;
+    const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
+    const float sc = 1.4426950408889634f * rsqrtf((float)kPfD);
+    float m = -INFINITY, l = 0.f, inv_l = 0.f;
+    uint32_t ph_s = 0, ph_o = 0;
+    bool ok = true;
+    float* probs = p.head_probs ? p.head_probs + (size_t)inst * p.num_visual : nullptr;
+    for (int pass = 0; pass < 2 && ok; ++pass) {
+      if (pass) inv_l = l > 0.f ? 1.f / l : 0.f;
+      for (int kt = 0; kt < nkt && ok; ++kt) {
+        ok = pf_wait(&bar_s, ph_s) && !*fail; ph_s ^= 1;
+        if (!ok) break;
+        tc_fence_after();
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {      // 32 key columns at a time
+          uint32_t v[32];
+          tmem_ld32(tmem_S + lane_addr + cb * 32, v);
+          const int j0 = kt * kTile + cb * 32;
+          if (!pass) {
+            float mx = m;
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+              const int j = j0 + c;
+              const float s = (j <= qi && j < T) ? __uint_as_float(v[c]) * sc : -INFINITY;
+              v[c] = __float_as_uint(s);
+              mx = fmaxf(mx, s);
+            }
+            if (mx > -INFINITY) {
+              float add = 0.f;
+#pragma unroll
+              for (int c = 0; c < 32; ++c) add += fast_exp2(__uint_as_float(v[c]) - mx);
+              l = l * fast_exp2(m - mx) + add;
+              m = mx;
+            }
+          } else {
+            // probabilities, as bf16, into the swizzled A-operand tile: 4 chunks of 8 keys
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                float pr[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                  const int c = ch * 8 + e * 2 + u;
+                  const int j = j0 + c;
+                  pr[u] = (live && j <= qi && j < T) ? fast_exp2(__uint_as_float(v[c]) * sc - m) * inv_l : 0.f;
+                  if (probs && qi == T - 1 && j >= p.sys_len && j < p.sys_len + p.num_visual) probs[j - p.sys_len] = pr[u];
+                }
+                const __nv_bfloat162 b2 = __floats2bfloat162_rn(pr[0], pr[1]);
+                w[e] = *reinterpret_cast<const uint32_t*>(&b2);
+              }
+              const int col = cb * 32 + ch * 8;               // first key of this 16-byte chunk
+              const int half = col >> 6, chunk = (col & 63) >> 3;
+              unsigned char* dst = sP + half * kBoxBytes + (r >> 3) * 1024 + (r & 7) * 128 + ((chunk ^ (r & 7)) << 4);
+              *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+        if (pass) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core
+        tc_fence_before();
+        mbar_arrive_cta(&bar_read);
+        if (pass) { ok = pf_wait(&bar_o, ph_o) && !*fail; ph_o ^= 1; }            // before P is overwritten
+      }
+    }
+    // ---- O (already normalised) -> bf16 -> global ----
+    if (ok) {
+      tc_fence_after();
+      __nv_bfloat16* orow = p.out + ((size_t)row_base + qi) * kPfD;
+#pragma unroll 1
+      for (int cb = 0; cb < 4; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tmem_O + lane_addr + cb * 32, v);
+        if (live) {
+#pragma unroll
+          for (int c = 0; c < 32; c += 8) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[c + 2 * e]), __uint_as_float(v[c + 2 * e + 1]));
+              w[e] = *reinterpret_cast<const uint32_t*>(&b2);
+            }
+            *reinterpret_cast<uint4*>(orow + cb * 32 + c) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+  }
+}
+
+// scores[b][i] = sum over the heads of sequence b of the last row's probability on visual token i
+__global__ void st3_prefill_scores_kernel(const float* __restrict__ head_probs, float* __restrict__ scores, int num_heads,
+                                          int num_visual) {
+  const int b = blockIdx.y;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= num_visual) return;
+  float s = 0.f;
+  for (int h = 0; h < num_heads; ++h) s += head_probs[((size_t)b * num_heads + h) * num_visual + i];
+  scores[(size_t)b * num_visual + i] = s;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// [rows][128] bf16 tensor, boxes of 128 rows x 64 columns, 128-byte swizzle, out-of-range rows read as zero.
+bool make_map(EncodeTiledFn fn, CUtensorMap* map, const void* base, size_t rows) {
+  const cuuint64_t dims[2] = {128, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {256};
+  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+extern "C" st3_status st3_prefill_attend(const void* q, const void* k, const void* v, void* out, float* head_probs,
+                                         float* scores, int* dev_status, int32_t num_inst, int32_t num_heads,
+                                         int32_t seq_len, int32_t head_dim, int32_t dtype, int32_t sys_len,
+                                         int32_t num_visual, void* cuda_stream) {
+  auto aligned = [](const void* ptr) { return ptr && (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; };
+  if (!aligned(q) || !aligned(k) || !aligned(v) || !aligned(out)) return ST3_ERR_INVALID_ARG;
+  if (num_inst < 1 || num_heads < 1 || num_inst % num_heads || seq_len < 1) return ST3_ERR_INVALID_ARG;
+  if (sys_len < 0 || num_visual < 0 || sys_len + num_visual > seq_len) return ST3_ERR_INVALID_ARG;
+  if (num_visual > 0 && (!head_probs || !scores)) return ST3_ERR_INVALID_ARG;
+  if (head_dim != kPfD || dtype != ST3_BF16) return ST3_ERR_UNSUPPORTED;
+  if ((long long)num_inst * seq_len > 0x7fffffffLL || num_inst > 65535) return ST3_ERR_UNSUPPORTED;
+  static EncodeTiledFn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess)
+      return ST3_ERR_CUDA;
+    encode = reinterpret_cast<EncodeTiledFn>(fn);
+  }
+  CUtensorMap mq, mk, mv;
+  const size_t rows = (size_t)num_inst * seq_len;
+  if (!make_map(encode, &mq, q, rows) || !make_map(encode, &mk, k, rows) || !make_map(encode, &mv, v, rows))
+    return ST3_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const int smem = 4 * kTileBytes2 + 1024;
+  if (cudaFuncSetAttribute(st3_prefill_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+    return ST3_ERR_CUDA;
+  PrefillParams p;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.head_probs = num_visual > 0 ? head_probs : nullptr;
+  p.status = dev_status;
+  p.T = seq_len; p.sys_len = sys_len; p.num_visual = num_visual;
+  const dim3 grid((unsigned)((seq_len + kTile - 1) / kTile), (unsigned)num_inst);
+  st3_prefill_attend_kernel<<<grid, kPfThreads, smem, st>>>(mq, mk, mv, p);
+  if (num_visual > 0) {
+    const dim3 g2((unsigned)((num_visual + 255) / 256), (unsigned)(num_inst / num_heads));
+    st3_prefill_scores_kernel<<<g2, 256, 0, st>>>(head_probs, scores, num_heads, num_visual);
+  }
+  return cudaGetLastError() == cudaSuccess ? ST3_OK : ST3_ERR_CUDA;
+}

@@ -98,10 +98,9 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   // the dynamic window is only 16-byte aligned by contract: round up to the 1024 bytes the swizzle needs
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* sQ = smem;
-  unsigned char* sK = sQ + kTileBytes2;
-  unsigned char* sV = sK + kTileBytes2;
-  unsigned char* sP = sV + kTileBytes2;
-  __shared__ __align__(8) uint64_t bar_q, bar_kv, bar_s, bar_read, bar_o;
+  unsigned char* sP = sQ + kTileBytes2;
+  unsigned char* sKV = sP + kTileBytes2;   // two buffers of [K tile | V tile]: the next key tile loads during this one
+  __shared__ __align__(8) uint64_t bar_q, bar_kv[2], bar_s, bar_read, bar_o;
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
 
@@ -112,7 +111,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   const int nkt = qt + 1;         // causal: key tiles 0..qt
 
   if (tid == 0) {
-    mbar_init(&bar_q, 1); mbar_init(&bar_kv, 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
+    mbar_init(&bar_q, 1); mbar_init(&bar_kv[0], 1); mbar_init(&bar_kv[1], 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
     mbar_init(&bar_read, 128);
     s_fail = 0;
     mbar_fence_init();
@@ -132,60 +131,68 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
 
   if (warp == 4) {
     // ===================== control warp =====================
-    uint32_t ph_kv = 0, ph_s = 0, ph_read = 0, ph_o = 0;
+    uint32_t ph_kv[2] = {0, 0}, ph_s = 0, ph_read = 0, ph_o = 0;
     bool ok = true;
+    const int nsteps = 2 * nkt;  // step = pass * nkt + key tile; step s uses K/V buffer s & 1
+    auto load_step = [&](int step) {
+      const int pass = step / nkt, kt = step - pass * nkt, buf = step & 1;
+      unsigned char* dK = sKV + buf * (2 * kTileBytes2);
+      unsigned char* dV = dK + kTileBytes2;
+      mbar_expect_tx(&bar_kv[buf], pass ? 2 * kTileBytes2 : kTileBytes2);
+      tma_load_2d(dK, &map_k, 0, row_base + kt * kTile, &bar_kv[buf]);
+      tma_load_2d(dK + kBoxBytes, &map_k, 64, row_base + kt * kTile, &bar_kv[buf]);
+      if (pass) {
+        tma_load_2d(dV, &map_v, 0, row_base + kt * kTile, &bar_kv[buf]);
+        tma_load_2d(dV + kBoxBytes, &map_v, 64, row_base + kt * kTile, &bar_kv[buf]);
+      }
+    };
     if (lane == 0) {
       mbar_expect_tx(&bar_q, kTileBytes2);
       tma_load_2d(sQ, &map_q, 0, row_base + qt * kTile, &bar_q);
       tma_load_2d(sQ + kBoxBytes, &map_q, 64, row_base + qt * kTile, &bar_q);
+      load_step(0);
     }
     ok = pf_wait(&bar_q, 0);
-    for (int pass = 0; pass < 2 && ok; ++pass) {
-      for (int kt = 0; kt < nkt && ok; ++kt) {
-        if (lane == 0) {
-          mbar_expect_tx(&bar_kv, pass ? 2 * kTileBytes2 : kTileBytes2);
-          tma_load_2d(sK, &map_k, 0, row_base + kt * kTile, &bar_kv);
-          tma_load_2d(sK + kBoxBytes, &map_k, 64, row_base + kt * kTile, &bar_kv);
-          if (pass) {
-            tma_load_2d(sV, &map_v, 0, row_base + kt * kTile, &bar_kv);
-            tma_load_2d(sV + kBoxBytes, &map_v, 64, row_base + kt * kTile, &bar_kv);
-          }
+    for (int step = 0; step < nsteps && ok; ++step) {
+      const int pass = step / nkt, kt = step - pass * nkt, buf = step & 1;
+      unsigned char* sK = sKV + buf * (2 * kTileBytes2);
+      unsigned char* sV = sK + kTileBytes2;
+      // the other buffer's last user (step - 1) has completed: fetch the next tile into it now
+      if (lane == 0 && step + 1 < nsteps) load_step(step + 1);
+      ok = pf_wait(&bar_kv[buf], ph_kv[buf]); ph_kv[buf] ^= 1;
+      if (!ok) break;
+      tc_fence_after();
+      if (lane == 0) {
+        // S = Q K^T: 8 steps of 16 along the head dimension
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
+          umma_bf16(tmem_S, smem_desc(smem_u32(sQ) + off, 16), smem_desc(smem_u32(sK) + off, 16), kIdescS, ks > 0);
         }
-        ok = pf_wait(&bar_kv, ph_kv); ph_kv ^= 1;
-        if (!ok) break;
+        umma_commit(&bar_s);
+      }
+      __syncwarp();
+      // the softmax warps have read S (pass 1) or have written P (pass 2)
+      ok = pf_wait(&bar_read, ph_read); ph_read ^= 1;
+      if (!ok) break;
+      if (pass) {
         tc_fence_after();
         if (lane == 0) {
-          // S = Q K^T: 8 steps of 16 along the head dimension
+          // O += P V: 8 steps of 16 keys; V is the MN-major operand (two 64-dim boxes 16 KB apart)
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
-            umma_bf16(tmem_S, smem_desc(smem_u32(sQ) + off, 16), smem_desc(smem_u32(sK) + off, 16), kIdescS, ks > 0);
+            const uint32_t offp = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
+            umma_bf16(tmem_O, smem_desc(smem_u32(sP) + offp, 16), smem_desc(smem_u32(sV) + ks * 2048, kBoxBytes),
+                      kIdescPV, (kt > 0 || ks > 0));
           }
-          umma_commit(&bar_s);
+          umma_commit(&bar_o);
         }
         __syncwarp();
-        // the softmax warps have read S (pass 1) or have written P (pass 2)
-        ok = pf_wait(&bar_read, ph_read); ph_read ^= 1;
-        if (!ok) break;
-        if (pass) {
-          tc_fence_after();
-          if (lane == 0) {
-            // O += P V: 8 steps of 16 keys; V is the MN-major operand (two 64-dim boxes 16 KB apart)
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-              const uint32_t offp = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
-              umma_bf16(tmem_O, smem_desc(smem_u32(sP) + offp, 16), smem_desc(smem_u32(sV) + ks * 2048, kBoxBytes),
-                        kIdescPV, (kt > 0 || ks > 0));
-            }
-            umma_commit(&bar_o);
-          }
-          __syncwarp();
-          ok = pf_wait(&bar_o, ph_o); ph_o ^= 1;   // K, V and P tiles are free again (and, at the end, O is complete)
-        } else {
-          ok = pf_wait(&bar_s, ph_s);              // the MMA is done with the K tile
-        }
-        ph_s ^= 1;
+        ok = pf_wait(&bar_o, ph_o); ph_o ^= 1;   // this buffer's K and V and the P tile are free again
+      } else {
+        ok = pf_wait(&bar_s, ph_s);              // the MMA is done with this buffer's K tile
       }
+      ph_s ^= 1;
     }
     if (!ok) { *fail = 1; if (lane == 0 && p.status) atomicOr(p.status, ST3_DEV_COPY_TIMEOUT); }
   } else {
@@ -340,7 +347,7 @@ extern "C" st3_status st3_prefill_attend(const void* q, const void* k, const voi
   if (!make_map(encode, &mq, q, rows) || !make_map(encode, &mk, k, rows) || !make_map(encode, &mv, v, rows))
     return ST3_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const int smem = 4 * kTileBytes2 + 1024;
+  const int smem = 6 * kTileBytes2 + 1024;   // Q, P, two [K | V] buffers
   if (cudaFuncSetAttribute(st3_prefill_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
     return ST3_ERR_CUDA;
   PrefillParams p;

@@ -346,6 +346,40 @@ def oracle_sample(wl, g, K, V, q0, q, kn, vn, nsteps, warm_steps, reps=1):
     return wl.batch * nsteps / secs, secs, threads, first, t - 1
 
 
+def prefill_attend_leg(wl, device, iters=10):
+    """Causal prompt attention (the step before the hot path) on the tensor cores: every layer's
+    (sequence, head) instances of the workload in one call, full prompt length."""
+    from paper_2412_20105_b200 import binding as B
+    if wl.dtype != "bf16" or wl.head_dim != 128:
+        return None
+    T = wl.sys_len + wl.num_visual + wl.text_len_max
+    n = min(wl.num_layers * wl.batch * wl.num_heads, 2048)
+    n -= n % wl.num_heads
+    g = torch.Generator().manual_seed(wl.seed)
+    mk = lambda: torch.randn(n, T, 128, generator=g).to(torch.bfloat16).to(device)
+    q, k, v = mk(), mk(), mk()
+    out = torch.empty_like(q)
+    probs = torch.zeros(n, wl.num_visual, device=device)
+    scores = torch.zeros(n // wl.num_heads, wl.num_visual, device=device)
+    st = torch.cuda.current_stream(device).cuda_stream
+    call = lambda: B.st3_prefill_attend(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), probs.data_ptr(),
+                                        scores.data_ptr(), None, n, wl.num_heads, T, 128, "bf16", wl.sys_len,
+                                        wl.num_visual, st)
+    for _ in range(3):
+        call()
+    ms = timed(call, iters, False) / iters
+    flops = n * 4 * 128 * T * (T + 1) / 2          # two GEMMs over the causal half
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak, src = float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        peak, src = 1590.0, "fallback"
+    tf = flops / (ms * 1e-3) / 1e12
+    return {"instances": n, "seq_len": T, "ms": ms, "bound": "tensor", "achieved": tf, "peak": peak,
+            "unit": "TFLOP/s", "frac": tf / peak, "peak_source": f"of {src}",
+            "flops": "causal half of Q K^T and P V (4 D T (T+1)/2 per instance); the kernel itself runs Q K^T twice"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -481,6 +515,7 @@ def main():
         job.ctx.status()
         line["per_layer_calls"] = {"value": tokens_per_gen * max(1, args.steps // 2) / (ms_pl * 1e-3), "unit": UNIT}
         line["kv_held"] = job.rows_held_curve()
+        line["prefill_attend"] = prefill_attend_leg(wl, device)
         # the oracle on the host cores, bounded sample
         ns = 24 if wl.batch == 1 else max(1, 24 // wl.batch)
         K, V, q0 = job.K.cpu(), job.V.cpu(), job.q0.cpu()

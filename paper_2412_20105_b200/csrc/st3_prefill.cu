@@ -1,10 +1,11 @@
 // Causal prompt attention (Eq. 2 in full) on the 5th-generation tensor cores: tcgen05.mma with
 // accumulators in tensor memory, operands staged in shared memory by TMA, for bf16 and D = 128.
 //
-// One block per (head instance, 128-query tile).  Warp 4 is the control warp: it issues the TMA loads
-// and the MMAs.  Warps 0-3 own one query row per thread (thread i <-> TMEM lane i), so the softmax needs
-// no cross-thread reduction.  Two passes over the key tiles 0..q_tile:
-//   pass 1   S = Q K^T (tcgen05.mma, 128x128x128), rows keep a running max and sum;
+// One block per (head instance, 128-query tile), two blocks per SM so that one block's softmax overlaps
+// the other's tensor work.  Warp 4 is the control warp: it issues the TMA loads and the MMAs.  Warps 0-3
+// own one query row per thread (thread i <-> TMEM lane i), so the softmax needs no cross-thread
+// reduction.  Two passes over the 64-key tiles up to the diagonal:
+//   pass 1   S = Q K^T (tcgen05.mma, 128x64x128), rows keep a running max and sum;
 //   pass 2   S again, P = exp2(S - max) / sum as bf16 into shared memory, O += P V (second MMA).
 // Recomputing S costs half again the tensor work but needs no rescaling of O in tensor memory.
 // The last query row's probabilities on the visual positions are written per head and summed over
@@ -20,11 +21,15 @@
 namespace {
 
 constexpr int kPfThreads = 160;       // 4 softmax warps + the control warp
-constexpr int kTile = 128;            // queries and keys per tile
+constexpr int kTile = 128;            // queries per tile
+constexpr int kKeys = 64;             // keys per tile
 constexpr int kPfD = 128;
-constexpr int kBoxBytes = 128 * 128;  // one TMA box: 128 rows x 64 bf16
+constexpr int kBoxBytes = 128 * 128;  // one TMA box of Q: 128 rows x 64 bf16
 constexpr int kTileBytes2 = 2 * kBoxBytes;
-constexpr uint32_t kTmemCols = 256;   // S in columns [0,128), O in [128,256)
+constexpr int kKBoxBytes = kKeys * 128;  // one TMA box of K or V: 64 rows x 64 bf16
+constexpr int kKTileBytes = 2 * kKBoxBytes;
+constexpr int kPBytes = kTile * kKeys * 2;  // probabilities of one tile, bf16
+constexpr uint32_t kTmemCols = 256;   // S in columns [0,64), O in [128,256)
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
   asm volatile(
@@ -79,10 +84,10 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// kind::f16 instruction descriptor: fp32 accumulate, bf16 x bf16, M = 128, N = 128.
-constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-constexpr uint32_t kIdescS = kIdescBase;               // A and B K-major
-constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);  // B (= V) MN-major
+// kind::f16 instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128.
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescS = kIdescBase | ((kKeys >> 3) << 17);                 // N = 64 keys, A and B K-major
+constexpr uint32_t kIdescPV = kIdescBase | ((128u >> 3) << 17) | (1u << 16);    // N = 128 dims, B (= V) MN-major
 
 struct PrefillParams {
   __nv_bfloat16* out;   // [num_inst][T][128]
@@ -91,7 +96,7 @@ struct PrefillParams {
   int T, sys_len, num_visual;
 };
 
-__global__ void __launch_bounds__(kPfThreads, 1)
+__global__ void __launch_bounds__(kPfThreads, 2)
 st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                           const __grid_constant__ CUtensorMap map_v, const PrefillParams p) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -99,8 +104,9 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* sQ = smem;
   unsigned char* sP = sQ + kTileBytes2;
-  unsigned char* sKV = sP + kTileBytes2;   // two buffers of [K tile | V tile]: the next key tile loads during this one
-  __shared__ __align__(8) uint64_t bar_q, bar_kv[2], bar_s, bar_read, bar_o;
+  unsigned char* sK = sP + kPBytes;
+  unsigned char* sV = sK + kKTileBytes;
+  __shared__ __align__(8) uint64_t bar_q, bar_kv, bar_s, bar_read, bar_o;
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
 
@@ -108,10 +114,10 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   const int qt = blockIdx.x, inst = blockIdx.y;
   const int T = p.T;
   const int row_base = inst * T;  // first row of this instance in the [num_inst * T][128] tensors
-  const int nkt = qt + 1;         // causal: key tiles 0..qt
+  const int nkt = (min(T, (qt + 1) * kTile) + kKeys - 1) / kKeys;  // causal: key tiles up to the diagonal
 
   if (tid == 0) {
-    mbar_init(&bar_q, 1); mbar_init(&bar_kv[0], 1); mbar_init(&bar_kv[1], 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
+    mbar_init(&bar_q, 1); mbar_init(&bar_kv, 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
     mbar_init(&bar_read, 128);
     s_fail = 0;
     mbar_fence_init();
@@ -131,68 +137,59 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
 
   if (warp == 4) {
     // ===================== control warp =====================
-    uint32_t ph_kv[2] = {0, 0}, ph_s = 0, ph_read = 0, ph_o = 0;
+    uint32_t ph_kv = 0, ph_s = 0, ph_read = 0, ph_o = 0;
     bool ok = true;
-    const int nsteps = 2 * nkt;  // step = pass * nkt + key tile; step s uses K/V buffer s & 1
-    auto load_step = [&](int step) {
-      const int pass = step / nkt, kt = step - pass * nkt, buf = step & 1;
-      unsigned char* dK = sKV + buf * (2 * kTileBytes2);
-      unsigned char* dV = dK + kTileBytes2;
-      mbar_expect_tx(&bar_kv[buf], pass ? 2 * kTileBytes2 : kTileBytes2);
-      tma_load_2d(dK, &map_k, 0, row_base + kt * kTile, &bar_kv[buf]);
-      tma_load_2d(dK + kBoxBytes, &map_k, 64, row_base + kt * kTile, &bar_kv[buf]);
-      if (pass) {
-        tma_load_2d(dV, &map_v, 0, row_base + kt * kTile, &bar_kv[buf]);
-        tma_load_2d(dV + kBoxBytes, &map_v, 64, row_base + kt * kTile, &bar_kv[buf]);
-      }
-    };
     if (lane == 0) {
       mbar_expect_tx(&bar_q, kTileBytes2);
       tma_load_2d(sQ, &map_q, 0, row_base + qt * kTile, &bar_q);
       tma_load_2d(sQ + kBoxBytes, &map_q, 64, row_base + qt * kTile, &bar_q);
-      load_step(0);
     }
     ok = pf_wait(&bar_q, 0);
-    for (int step = 0; step < nsteps && ok; ++step) {
-      const int pass = step / nkt, kt = step - pass * nkt, buf = step & 1;
-      unsigned char* sK = sKV + buf * (2 * kTileBytes2);
-      unsigned char* sV = sK + kTileBytes2;
-      // the other buffer's last user (step - 1) has completed: fetch the next tile into it now
-      if (lane == 0 && step + 1 < nsteps) load_step(step + 1);
-      ok = pf_wait(&bar_kv[buf], ph_kv[buf]); ph_kv[buf] ^= 1;
-      if (!ok) break;
-      tc_fence_after();
-      if (lane == 0) {
-        // S = Q K^T: 8 steps of 16 along the head dimension
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t off = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
-          umma_bf16(tmem_S, smem_desc(smem_u32(sQ) + off, 16), smem_desc(smem_u32(sK) + off, 16), kIdescS, ks > 0);
+    for (int pass = 0; pass < 2 && ok; ++pass) {
+      for (int kt = 0; kt < nkt && ok; ++kt) {
+        if (lane == 0) {
+          mbar_expect_tx(&bar_kv, pass ? 2 * kKTileBytes : kKTileBytes);
+          tma_load_2d(sK, &map_k, 0, row_base + kt * kKeys, &bar_kv);
+          tma_load_2d(sK + kKBoxBytes, &map_k, 64, row_base + kt * kKeys, &bar_kv);
+          if (pass) {
+            tma_load_2d(sV, &map_v, 0, row_base + kt * kKeys, &bar_kv);
+            tma_load_2d(sV + kKBoxBytes, &map_v, 64, row_base + kt * kKeys, &bar_kv);
+          }
         }
-        umma_commit(&bar_s);
-      }
-      __syncwarp();
-      // the softmax warps have read S (pass 1) or have written P (pass 2)
-      ok = pf_wait(&bar_read, ph_read); ph_read ^= 1;
-      if (!ok) break;
-      if (pass) {
+        ok = pf_wait(&bar_kv, ph_kv); ph_kv ^= 1;
+        if (!ok) break;
         tc_fence_after();
         if (lane == 0) {
-          // O += P V: 8 steps of 16 keys; V is the MN-major operand (two 64-dim boxes 16 KB apart)
+          // S = Q K^T: 8 steps of 16 along the head dimension
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t offp = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
-            umma_bf16(tmem_O, smem_desc(smem_u32(sP) + offp, 16), smem_desc(smem_u32(sV) + ks * 2048, kBoxBytes),
-                      kIdescPV, (kt > 0 || ks > 0));
+            const uint32_t offq = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
+            const uint32_t offk = (ks >> 2) * kKBoxBytes + (ks & 3) * 32;
+            umma_bf16(tmem_S, smem_desc(smem_u32(sQ) + offq, 16), smem_desc(smem_u32(sK) + offk, 16), kIdescS, ks > 0);
           }
-          umma_commit(&bar_o);
+          umma_commit(&bar_s);
         }
         __syncwarp();
-        ok = pf_wait(&bar_o, ph_o); ph_o ^= 1;   // this buffer's K and V and the P tile are free again
-      } else {
-        ok = pf_wait(&bar_s, ph_s);              // the MMA is done with this buffer's K tile
+        // the softmax warps have read S (pass 1) or have written P (pass 2)
+        ok = pf_wait(&bar_read, ph_read); ph_read ^= 1;
+        if (!ok) break;
+        if (pass) {
+          tc_fence_after();
+          if (lane == 0) {
+            // O += P V: 4 steps of 16 keys; V is the MN-major operand (two 64-dim boxes 8 KB apart)
+#pragma unroll
+            for (int ks = 0; ks < kKeys / 16; ++ks)
+              umma_bf16(tmem_O, smem_desc(smem_u32(sP) + ks * 32, 16), smem_desc(smem_u32(sV) + ks * 2048, kKBoxBytes),
+                        kIdescPV, (kt > 0 || ks > 0));
+            umma_commit(&bar_o);
+          }
+          __syncwarp();
+          ok = pf_wait(&bar_o, ph_o); ph_o ^= 1;   // K, V and P tiles are free again (and, at the end, O is complete)
+        } else {
+          ok = pf_wait(&bar_s, ph_s);              // the MMA is done with the K tile
+        }
+        ph_s ^= 1;
       }
-      ph_s ^= 1;
     }
     if (!ok) { *fail = 1; if (lane == 0 && p.status) atomicOr(p.status, ST3_DEV_COPY_TIMEOUT); }
   } else {
@@ -213,10 +210,10 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
         if (!ok) break;
         tc_fence_after();
 #pragma unroll 1
-        for (int cb = 0; cb < 4; ++cb) {      // 32 key columns at a time
+        for (int cb = 0; cb < kKeys / 32; ++cb) {      // 32 key columns at a time
           uint32_t v[32];
           tmem_ld32(tmem_S + lane_addr + cb * 32, v);
-          const int j0 = kt * kTile + cb * 32;
+          const int j0 = kt * kKeys + cb * 32;
           if (!pass) {
             float mx = m;
 #pragma unroll
@@ -251,9 +248,8 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                 const __nv_bfloat162 b2 = __floats2bfloat162_rn(pr[0], pr[1]);
                 w[e] = *reinterpret_cast<const uint32_t*>(&b2);
               }
-              const int col = cb * 32 + ch * 8;               // first key of this 16-byte chunk
-              const int half = col >> 6, chunk = (col & 63) >> 3;
-              unsigned char* dst = sP + half * kBoxBytes + (r >> 3) * 1024 + (r & 7) * 128 + ((chunk ^ (r & 7)) << 4);
+              const int chunk = cb * 4 + ch;                  // which 16-byte chunk (8 keys) of the 128-byte row
+              unsigned char* dst = sP + (r >> 3) * 1024 + (r & 7) * 128 + ((chunk ^ (r & 7)) << 4);
               *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
             }
           }
@@ -309,11 +305,11 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// [rows][128] bf16 tensor, boxes of 128 rows x 64 columns, 128-byte swizzle, out-of-range rows read as zero.
-bool make_map(EncodeTiledFn fn, CUtensorMap* map, const void* base, size_t rows) {
+// [rows][128] bf16 tensor, boxes of box_rows rows x 64 columns, 128-byte swizzle, out-of-range rows read as zero.
+bool make_map(EncodeTiledFn fn, CUtensorMap* map, const void* base, size_t rows, int box_rows) {
   const cuuint64_t dims[2] = {128, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {256};
-  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -344,10 +340,11 @@ extern "C" st3_status st3_prefill_attend(const void* q, const void* k, const voi
   }
   CUtensorMap mq, mk, mv;
   const size_t rows = (size_t)num_inst * seq_len;
-  if (!make_map(encode, &mq, q, rows) || !make_map(encode, &mk, k, rows) || !make_map(encode, &mv, v, rows))
+  if (!make_map(encode, &mq, q, rows, kTile) || !make_map(encode, &mk, k, rows, kKeys) ||
+      !make_map(encode, &mv, v, rows, kKeys))
     return ST3_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const int smem = 6 * kTileBytes2 + 1024;   // Q, P, two [K | V] buffers
+  const int smem = kTileBytes2 + kPBytes + 2 * kKTileBytes + 1024;   // Q, P, K, V (+ alignment slack)
   if (cudaFuncSetAttribute(st3_prefill_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
     return ST3_ERR_CUDA;
   PrefillParams p;

@@ -4,12 +4,13 @@
 // One block per (head instance, 128-query tile), two blocks per SM so that one block's softmax overlaps
 // the other's tensor work.  Warp 4 is the control warp: it issues the TMA loads and the MMAs.  Warps 0-3
 // own one query row per thread (thread i <-> TMEM lane i), so the softmax needs no cross-thread
-// reduction.  Two passes over the 64-key tiles up to the diagonal:
-//   pass 1   S = Q K^T (tcgen05.mma, 128x64x128), rows keep a running max and sum;
-//   pass 2   S again, P = exp2(S - max) / sum as bf16 into shared memory, O += P V (second MMA).
-// Recomputing S costs half again the tensor work but needs no rescaling of O in tensor memory.
-// The last query row's probabilities on the visual positions are written per head and summed over
-// heads by a second small kernel: the scores alpha (Sec. 3.2) that prune the NEXT layer.
+// reduction.  One pass over the 64-key tiles up to the diagonal, with an online softmax:
+//   S = Q K^T (tcgen05.mma, 128x64x128); P = exp2(S - ref) as bf16 into shared memory; O += P V (second
+//   MMA, accumulator in tensor memory).  `ref` follows the row's running maximum lazily: O (and the running
+//   sum) are rescaled in tensor memory only when the maximum has grown by more than 2^8, so P never
+//   exceeds 256 and rescaling is rare after the first tiles; O is divided by the sum on the way out.
+// The last query row's logits on the visual positions are kept per head, normalised at the end and summed
+// over heads by a second small kernel: the scores alpha (Sec. 3.2) that prune the NEXT layer.
 //
 // Shared-memory operand layout: 128-byte swizzle, K-major tiles of [rows][64 bf16] (what a TMA box with
 // CU_TENSOR_MAP_SWIZZLE_128B writes); V is consumed as an MN-major B operand straight from the same
@@ -81,6 +82,17 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "memory");
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+      "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+      "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+  asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -137,7 +149,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
 
   if (warp == 4) {
     // ===================== control warp =====================
-    uint32_t ph_kv = 0, ph_s = 0, ph_read = 0, ph_o = 0;
+    uint32_t ph_kv = 0, ph_read = 0, ph_o = 0;
     bool ok = true;
     if (lane == 0) {
       mbar_expect_tx(&bar_q, kTileBytes2);
@@ -145,51 +157,42 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       tma_load_2d(sQ + kBoxBytes, &map_q, 64, row_base + qt * kTile, &bar_q);
     }
     ok = pf_wait(&bar_q, 0);
-    for (int pass = 0; pass < 2 && ok; ++pass) {
-      for (int kt = 0; kt < nkt && ok; ++kt) {
-        if (lane == 0) {
-          mbar_expect_tx(&bar_kv, pass ? 2 * kKTileBytes : kKTileBytes);
-          tma_load_2d(sK, &map_k, 0, row_base + kt * kKeys, &bar_kv);
-          tma_load_2d(sK + kKBoxBytes, &map_k, 64, row_base + kt * kKeys, &bar_kv);
-          if (pass) {
-            tma_load_2d(sV, &map_v, 0, row_base + kt * kKeys, &bar_kv);
-            tma_load_2d(sV + kKBoxBytes, &map_v, 64, row_base + kt * kKeys, &bar_kv);
-          }
-        }
-        ok = pf_wait(&bar_kv, ph_kv); ph_kv ^= 1;
-        if (!ok) break;
-        tc_fence_after();
-        if (lane == 0) {
-          // S = Q K^T: 8 steps of 16 along the head dimension
-#pragma unroll
-          for (int ks = 0; ks < 8; ++ks) {
-            const uint32_t offq = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
-            const uint32_t offk = (ks >> 2) * kKBoxBytes + (ks & 3) * 32;
-            umma_bf16(tmem_S, smem_desc(smem_u32(sQ) + offq, 16), smem_desc(smem_u32(sK) + offk, 16), kIdescS, ks > 0);
-          }
-          umma_commit(&bar_s);
-        }
-        __syncwarp();
-        // the softmax warps have read S (pass 1) or have written P (pass 2)
-        ok = pf_wait(&bar_read, ph_read); ph_read ^= 1;
-        if (!ok) break;
-        if (pass) {
-          tc_fence_after();
-          if (lane == 0) {
-            // O += P V: 4 steps of 16 keys; V is the MN-major operand (two 64-dim boxes 8 KB apart)
-#pragma unroll
-            for (int ks = 0; ks < kKeys / 16; ++ks)
-              umma_bf16(tmem_O, smem_desc(smem_u32(sP) + ks * 32, 16), smem_desc(smem_u32(sV) + ks * 2048, kKBoxBytes),
-                        kIdescPV, (kt > 0 || ks > 0));
-            umma_commit(&bar_o);
-          }
-          __syncwarp();
-          ok = pf_wait(&bar_o, ph_o); ph_o ^= 1;   // K, V and P tiles are free again (and, at the end, O is complete)
-        } else {
-          ok = pf_wait(&bar_s, ph_s);              // the MMA is done with the K tile
-        }
-        ph_s ^= 1;
+    for (int kt = 0; kt < nkt && ok; ++kt) {
+      if (lane == 0) {
+        mbar_expect_tx(&bar_kv, 2 * kKTileBytes);
+        tma_load_2d(sK, &map_k, 0, row_base + kt * kKeys, &bar_kv);
+        tma_load_2d(sK + kKBoxBytes, &map_k, 64, row_base + kt * kKeys, &bar_kv);
+        tma_load_2d(sV, &map_v, 0, row_base + kt * kKeys, &bar_kv);
+        tma_load_2d(sV + kKBoxBytes, &map_v, 64, row_base + kt * kKeys, &bar_kv);
       }
+      ok = pf_wait(&bar_kv, ph_kv); ph_kv ^= 1;
+      if (!ok) break;
+      tc_fence_after();
+      if (lane == 0) {
+        // S = Q K^T: 8 steps of 16 along the head dimension
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t offq = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
+          const uint32_t offk = (ks >> 2) * kKBoxBytes + (ks & 3) * 32;
+          umma_bf16(tmem_S, smem_desc(smem_u32(sQ) + offq, 16), smem_desc(smem_u32(sK) + offk, 16), kIdescS, ks > 0);
+        }
+        umma_commit(&bar_s);
+      }
+      __syncwarp();
+      // the softmax warps have read S, rescaled O if they had to, and written P
+      ok = pf_wait(&bar_read, ph_read); ph_read ^= 1;
+      if (!ok) break;
+      tc_fence_after();
+      if (lane == 0) {
+        // O += P V: 4 steps of 16 keys; V is the MN-major operand (two 64-dim boxes 8 KB apart)
+#pragma unroll
+        for (int ks = 0; ks < kKeys / 16; ++ks)
+          umma_bf16(tmem_O, smem_desc(smem_u32(sP) + ks * 32, 16), smem_desc(smem_u32(sV) + ks * 2048, kKBoxBytes),
+                    kIdescPV, (kt > 0 || ks > 0));
+        umma_commit(&bar_o);
+      }
+      __syncwarp();
+      ok = pf_wait(&bar_o, ph_o); ph_o ^= 1;   // K, V and P tiles are free again (and, at the end, O is complete)
     }
     if (!ok) { *fail = 1; if (lane == 0 && p.status) atomicOr(p.status, ST3_DEV_COPY_TIMEOUT); }
   } else {
@@ -199,68 +202,84 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     const bool live = qi < T;
     const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
     const float sc = 1.4426950408889634f * rsqrtf((float)kPfD);
-    float m = -INFINITY, l = 0.f, inv_l = 0.f;
+    float ref = -INFINITY;   // what P is taken relative to; trails the running maximum by at most 8 (log2 domain)
+    float l = 0.f;           // running sum of exp2(s - ref)
     uint32_t ph_s = 0, ph_o = 0;
     bool ok = true;
     float* probs = p.head_probs ? p.head_probs + (size_t)inst * p.num_visual : nullptr;
-    for (int pass = 0; pass < 2 && ok; ++pass) {
-      if (pass) inv_l = l > 0.f ? 1.f / l : 0.f;
-      for (int kt = 0; kt < nkt && ok; ++kt) {
-        ok = pf_wait(&bar_s, ph_s) && !*fail; ph_s ^= 1;
-        if (!ok) break;
-        tc_fence_after();
-#pragma unroll 1
-        for (int cb = 0; cb < kKeys / 32; ++cb) {      // 32 key columns at a time
-          uint32_t v[32];
-          tmem_ld32(tmem_S + lane_addr + cb * 32, v);
-          const int j0 = kt * kKeys + cb * 32;
-          if (!pass) {
-            float mx = m;
+    const bool last_row = live && qi == T - 1;
+    for (int kt = 0; kt < nkt && ok; ++kt) {
+      ok = pf_wait(&bar_s, ph_s) && !*fail; ph_s ^= 1;
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t v0[32], v1[32];
+      tmem_ld32(tmem_S + lane_addr, v0);
+      tmem_ld32(tmem_S + lane_addr + 32, v1);
+      const int j0 = kt * kKeys;
+      float mx = -INFINITY;
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-              const int j = j0 + c;
-              const float s = (j <= qi && j < T) ? __uint_as_float(v[c]) * sc : -INFINITY;
-              v[c] = __float_as_uint(s);
-              mx = fmaxf(mx, s);
-            }
-            if (mx > -INFINITY) {
-              float add = 0.f;
-#pragma unroll
-              for (int c = 0; c < 32; ++c) add += fast_exp2(__uint_as_float(v[c]) - mx);
-              l = l * fast_exp2(m - mx) + add;
-              m = mx;
-            }
-          } else {
-            // probabilities, as bf16, into the swizzled A-operand tile: 4 chunks of 8 keys
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-              uint32_t w[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                float pr[2];
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                  const int c = ch * 8 + e * 2 + u;
-                  const int j = j0 + c;
-                  pr[u] = (live && j <= qi && j < T) ? fast_exp2(__uint_as_float(v[c]) * sc - m) * inv_l : 0.f;
-                  if (probs && qi == T - 1 && j >= p.sys_len && j < p.sys_len + p.num_visual) probs[j - p.sys_len] = pr[u];
-                }
-                const __nv_bfloat162 b2 = __floats2bfloat162_rn(pr[0], pr[1]);
-                w[e] = *reinterpret_cast<const uint32_t*>(&b2);
-              }
-              const int chunk = cb * 4 + ch;                  // which 16-byte chunk (8 keys) of the 128-byte row
-              unsigned char* dst = sP + (r >> 3) * 1024 + (r & 7) * 128 + ((chunk ^ (r & 7)) << 4);
-              *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-          }
-        }
-        if (pass) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core
-        tc_fence_before();
-        mbar_arrive_cta(&bar_read);
-        if (pass) { ok = pf_wait(&bar_o, ph_o) && !*fail; ph_o ^= 1; }            // before P is overwritten
+      for (int c = 0; c < 32; ++c) {
+        const float s0 = (live && j0 + c <= qi && j0 + c < T) ? __uint_as_float(v0[c]) * sc : -INFINITY;
+        const float s1 = (live && j0 + 32 + c <= qi && j0 + 32 + c < T) ? __uint_as_float(v1[c]) * sc : -INFINITY;
+        v0[c] = __float_as_uint(s0); v1[c] = __float_as_uint(s1);
+        mx = fmaxf(mx, fmaxf(s0, s1));
       }
+      if (last_row && probs) {   // the logits of the visual positions; normalised once the row is complete
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          const int ja = j0 + c - p.sys_len, jb = ja + 32;
+          if (ja >= 0 && ja < p.num_visual) probs[ja] = __uint_as_float(v0[c]);
+          if (jb >= 0 && jb < p.num_visual) probs[jb] = __uint_as_float(v1[c]);
+        }
+      }
+      // lazy rescale: move the reference only when the maximum has run away from it
+      float factor = 1.f;
+      if (mx > ref + 8.f) {
+        factor = ref > -INFINITY ? fast_exp2(ref - mx) : 0.f;
+        ref = mx;
+      }
+      if (kt > 0 && __any_sync(0xffffffffu, factor != 1.f)) {
+        // the previous P V has completed (bar_o was waited below), so O is stable: scale this row in place
+#pragma unroll 1
+        for (int cb = 0; cb < 4; ++cb) {
+          uint32_t o[32];
+          tmem_ld32(tmem_O + lane_addr + cb * 32, o);
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * factor);
+          tmem_st32(tmem_O + lane_addr + cb * 32, o);
+        }
+      }
+      l *= factor;
+      // probabilities, as bf16, into the swizzled A-operand tile: 8 chunks of 8 keys
+      const float rf = ref > -INFINITY ? ref : 0.f;   // a row with no key yet (padding rows) yields zeros
+      float add = 0.f;
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int c = (ch & 3) * 8 + e * 2;
+          const float sa = __uint_as_float(ch < 4 ? v0[c] : v1[c]), sb = __uint_as_float(ch < 4 ? v0[c + 1] : v1[c + 1]);
+          const float pa = fast_exp2(sa - rf), pb = fast_exp2(sb - rf);   // exp2(-inf) = 0 for masked keys
+          add += pa + pb;
+          const __nv_bfloat162 b2 = __floats2bfloat162_rn(pa, pb);
+          w[e] = *reinterpret_cast<const uint32_t*>(&b2);
+        }
+        unsigned char* dst = sP + (r >> 3) * 1024 + (r & 7) * 128 + ((ch ^ (r & 7)) << 4);
+        *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      l += add;
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core
+      tc_fence_before();
+      mbar_arrive_cta(&bar_read);
+      ok = pf_wait(&bar_o, ph_o) && !*fail; ph_o ^= 1;               // P V done: P may be overwritten, O is stable
     }
-    // ---- O (already normalised) -> bf16 -> global ----
+    const float inv_l = l > 0.f ? 1.f / l : 0.f;
+    if (ok && last_row && probs) {
+      // alpha of this head: exp2(logit - ref) / sum over the visual positions (ref is final here)
+      for (int i = 0; i < p.num_visual; ++i) probs[i] = fast_exp2(probs[i] - ref) * inv_l;
+    }
+    // ---- O / sum -> bf16 -> global ----
     if (ok) {
       tc_fence_after();
       __nv_bfloat16* orow = p.out + ((size_t)row_base + qi) * kPfD;
@@ -274,7 +293,8 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
             uint32_t w[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[c + 2 * e]), __uint_as_float(v[c + 2 * e + 1]));
+              const __nv_bfloat162 b2 = __floats2bfloat162_rn(__uint_as_float(v[c + 2 * e]) * inv_l,
+                                                              __uint_as_float(v[c + 2 * e + 1]) * inv_l);
               w[e] = *reinterpret_cast<const uint32_t*>(&b2);
             }
             *reinterpret_cast<uint4*>(orow + cb * 32 + c) = make_uint4(w[0], w[1], w[2], w[3]);

@@ -121,6 +121,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   __shared__ __align__(8) uint64_t bar_q, bar_kv, bar_s, bar_read, bar_o;
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
+  __shared__ float s_last[2];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int qt = blockIdx.x, inst = blockIdx.y;
@@ -275,9 +276,14 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       ok = pf_wait(&bar_o, ph_o) && !*fail; ph_o ^= 1;               // P V done: P may be overwritten, O is stable
     }
     const float inv_l = l > 0.f ? 1.f / l : 0.f;
-    if (ok && last_row && probs) {
-      // alpha of this head: exp2(logit - ref) / sum over the visual positions (ref is final here)
-      for (int i = 0; i < p.num_visual; ++i) probs[i] = fast_exp2(probs[i] - ref) * inv_l;
+    if (probs && (T - 1) / kTile == qt) {   // this block holds the last query row (same answer in every thread)
+      // alpha of this head: exp2(logit - ref) / sum over the visual positions, with the last row's final
+      // reference and sum; the 128 softmax threads share the work
+      if (last_row) { s_last[0] = ref; s_last[1] = ok ? inv_l : 0.f; }
+      __threadfence_block();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      const float rl = s_last[0], il = s_last[1];
+      for (int i = tid; i < p.num_visual; i += 128) probs[i] = fast_exp2(probs[i] - rl) * il;
     }
     // ---- O / sum -> bf16 -> global ----
     if (ok) {

@@ -377,7 +377,7 @@ def prefill_attend_leg(wl, device, iters=10):
     tf = flops / (ms * 1e-3) / 1e12
     return {"instances": n, "seq_len": T, "ms": ms, "bound": "tensor", "achieved": tf, "peak": peak,
             "unit": "TFLOP/s", "frac": tf / peak, "peak_source": f"of {src}",
-            "flops": "causal half of Q K^T and P V (4 D T (T+1)/2 per instance); the kernel itself runs Q K^T twice"}
+            "flops": "causal half of Q K^T and P V (4 D T (T+1)/2 per instance)"}
 
 
 def main():

@@ -116,9 +116,9 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* sQ = smem;
   unsigned char* sP = sQ + kTileBytes2;
-  unsigned char* sK = sP + kPBytes;
-  unsigned char* sV = sK + kKTileBytes;
-  __shared__ __align__(8) uint64_t bar_q, bar_kv, bar_s, bar_read, bar_o;
+  unsigned char* sV = sP + kPBytes;
+  unsigned char* sK2 = sV + kKTileBytes;   // two K buffers: tile t+2 replaces tile t as soon as S(t) is complete
+  __shared__ __align__(8) uint64_t bar_q, bar_k[2], bar_v, bar_s[2], bar_p, bar_o;
   __shared__ uint32_t s_tmem;
   __shared__ int s_fail;
   __shared__ float s_last[2];
@@ -130,8 +130,9 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   const int nkt = (min(T, (qt + 1) * kTile) + kKeys - 1) / kKeys;  // causal: key tiles up to the diagonal
 
   if (tid == 0) {
-    mbar_init(&bar_q, 1); mbar_init(&bar_kv, 1); mbar_init(&bar_s, 1); mbar_init(&bar_o, 1);
-    mbar_init(&bar_read, 128);
+    mbar_init(&bar_q, 1); mbar_init(&bar_k[0], 1); mbar_init(&bar_k[1], 1); mbar_init(&bar_v, 1);
+    mbar_init(&bar_s[0], 1); mbar_init(&bar_s[1], 1); mbar_init(&bar_o, 1);
+    mbar_init(&bar_p, 128);
     s_fail = 0;
     mbar_fence_init();
   }
@@ -145,44 +146,66 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = s_tmem;
-  const uint32_t tmem_S = tmem, tmem_O = tmem + 128;
+  const uint32_t tmem_O = tmem + 128;   // S(t) lives at column 64 * (t & 1)
   volatile int* fail = &s_fail;
 
   if (warp == 4) {
     // ===================== control warp =====================
-    uint32_t ph_kv = 0, ph_read = 0, ph_o = 0;
+    // Tensor-pipe order: S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...  -- S(t+1) is already in tensor memory when
+    // the softmax of tile t ends, so the softmax warps never wait for the tensor cores in steady state.
     bool ok = true;
+    auto load_k = [&](int kt) {
+      unsigned char* d = sK2 + (kt & 1) * kKTileBytes;
+      mbar_expect_tx(&bar_k[kt & 1], kKTileBytes);
+      tma_load_2d(d, &map_k, 0, row_base + kt * kKeys, &bar_k[kt & 1]);
+      tma_load_2d(d + kKBoxBytes, &map_k, 64, row_base + kt * kKeys, &bar_k[kt & 1]);
+    };
+    auto load_v = [&](int kt) {
+      mbar_expect_tx(&bar_v, kKTileBytes);
+      tma_load_2d(sV, &map_v, 0, row_base + kt * kKeys, &bar_v);
+      tma_load_2d(sV + kKBoxBytes, &map_v, 64, row_base + kt * kKeys, &bar_v);
+    };
+    // S(kt) = Q K(kt)^T: 8 steps of 16 along the head dimension
+    auto issue_s = [&](int kt) {
+      const unsigned char* sK = sK2 + (kt & 1) * kKTileBytes;
+      const uint32_t tmem_S = tmem + (uint32_t)(kt & 1) * kKeys;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        const uint32_t offq = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
+        const uint32_t offk = (ks >> 2) * kKBoxBytes + (ks & 3) * 32;
+        umma_bf16(tmem_S, smem_desc(smem_u32(sQ) + offq, 16), smem_desc(smem_u32(sK) + offk, 16), kIdescS, ks > 0);
+      }
+      umma_commit(&bar_s[kt & 1]);
+    };
     if (lane == 0) {
       mbar_expect_tx(&bar_q, kTileBytes2);
       tma_load_2d(sQ, &map_q, 0, row_base + qt * kTile, &bar_q);
       tma_load_2d(sQ + kBoxBytes, &map_q, 64, row_base + qt * kTile, &bar_q);
+      load_k(0);
+      if (nkt > 1) load_k(1);
+      load_v(0);
     }
     ok = pf_wait(&bar_q, 0);
-    for (int kt = 0; kt < nkt && ok; ++kt) {
-      if (lane == 0) {
-        mbar_expect_tx(&bar_kv, 2 * kKTileBytes);
-        tma_load_2d(sK, &map_k, 0, row_base + kt * kKeys, &bar_kv);
-        tma_load_2d(sK + kKBoxBytes, &map_k, 64, row_base + kt * kKeys, &bar_kv);
-        tma_load_2d(sV, &map_v, 0, row_base + kt * kKeys, &bar_kv);
-        tma_load_2d(sV + kKBoxBytes, &map_v, 64, row_base + kt * kKeys, &bar_kv);
-      }
-      ok = pf_wait(&bar_kv, ph_kv); ph_kv ^= 1;
+    // prologue: S(0) and S(1); then K(2), K(3) into the buffers they leave
+    for (int kt = 0; kt < 2 && kt < nkt && ok; ++kt) {
+      ok = pf_wait(&bar_k[kt], 0);
       if (!ok) break;
       tc_fence_after();
-      if (lane == 0) {
-        // S = Q K^T: 8 steps of 16 along the head dimension
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t offq = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
-          const uint32_t offk = (ks >> 2) * kKBoxBytes + (ks & 3) * 32;
-          umma_bf16(tmem_S, smem_desc(smem_u32(sQ) + offq, 16), smem_desc(smem_u32(sK) + offk, 16), kIdescS, ks > 0);
-        }
-        umma_commit(&bar_s);
-      }
+      if (lane == 0) issue_s(kt);
       __syncwarp();
-      // the softmax warps have read S, rescaled O if they had to, and written P
-      ok = pf_wait(&bar_read, ph_read); ph_read ^= 1;
+    }
+    for (int kt = 0; kt < 2 && kt + 2 < nkt && ok; ++kt) {
+      ok = pf_wait(&bar_s[kt], 0);
+      if (ok && lane == 0) load_k(kt + 2);
+      __syncwarp();
+    }
+    for (int kt = 0; kt < nkt && ok; ++kt) {
+      // P(kt) is in shared memory (its writers have also seen P V(kt-1) complete) and V(kt) has landed
+      ok = pf_wait(&bar_p, kt & 1);
       if (!ok) break;
+      ok = pf_wait(&bar_v, kt & 1);
+      if (!ok) break;
+      if (kt + 2 < nkt) { ok = pf_wait(&bar_k[kt & 1], ((kt + 2) >> 1) & 1); if (!ok) break; }
       tc_fence_after();
       if (lane == 0) {
         // O += P V: 4 steps of 16 keys; V is the MN-major operand (two 64-dim boxes 8 KB apart)
@@ -191,9 +214,19 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
           umma_bf16(tmem_O, smem_desc(smem_u32(sP) + ks * 32, 16), smem_desc(smem_u32(sV) + ks * 2048, kKBoxBytes),
                     kIdescPV, (kt > 0 || ks > 0));
         umma_commit(&bar_o);
+        if (kt + 2 < nkt) issue_s(kt + 2);   // into the S buffer whose tile the softmax warps have just left
       }
       __syncwarp();
-      ok = pf_wait(&bar_o, ph_o); ph_o ^= 1;   // K, V and P tiles are free again (and, at the end, O is complete)
+      // refill what these MMAs release: V's buffer after P V(kt), K's buffer after S(kt+2)
+      ok = pf_wait(&bar_o, kt & 1);
+      if (!ok) break;
+      if (lane == 0 && kt + 1 < nkt) load_v(kt + 1);
+      if (kt + 4 < nkt) {
+        ok = pf_wait(&bar_s[kt & 1], ((kt + 2) >> 1) & 1);
+        if (!ok) break;
+        if (lane == 0) load_k(kt + 4);
+      }
+      __syncwarp();
     }
     if (!ok) { *fail = 1; if (lane == 0 && p.status) atomicOr(p.status, ST3_DEV_COPY_TIMEOUT); }
   } else {
@@ -205,32 +238,35 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     const float sc = 1.4426950408889634f * rsqrtf((float)kPfD);
     float ref = -INFINITY;   // what P is taken relative to; trails the running maximum by at most 8 (log2 domain)
     float l = 0.f;           // running sum of exp2(s - ref)
-    uint32_t ph_s = 0, ph_o = 0;
     bool ok = true;
     float* probs = p.head_probs ? p.head_probs + (size_t)inst * p.num_visual : nullptr;
     const bool last_row = live && qi == T - 1;
     for (int kt = 0; kt < nkt && ok; ++kt) {
-      ok = pf_wait(&bar_s, ph_s) && !*fail; ph_s ^= 1;
+      ok = pf_wait(&bar_s[kt & 1], (kt >> 1) & 1) && !*fail;
       if (!ok) break;
       tc_fence_after();
+      const uint32_t tmem_S = tmem + (uint32_t)(kt & 1) * kKeys;
       uint32_t v0[32], v1[32];
       tmem_ld32(tmem_S + lane_addr, v0);
       tmem_ld32(tmem_S + lane_addr + 32, v1);
       const int j0 = kt * kKeys;
+      if (j0 + kKeys > qt * kTile + 1 || j0 + kKeys > T) {   // the tile touches the diagonal or the end of the prompt
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          if (!(live && j0 + c <= qi && j0 + c < T)) v0[c] = 0xff800000u;
+          if (!(live && j0 + 32 + c <= qi && j0 + 32 + c < T)) v1[c] = 0xff800000u;
+        }
+      }
       float mx = -INFINITY;
 #pragma unroll
-      for (int c = 0; c < 32; ++c) {
-        const float s0 = (live && j0 + c <= qi && j0 + c < T) ? __uint_as_float(v0[c]) * sc : -INFINITY;
-        const float s1 = (live && j0 + 32 + c <= qi && j0 + 32 + c < T) ? __uint_as_float(v1[c]) * sc : -INFINITY;
-        v0[c] = __float_as_uint(s0); v1[c] = __float_as_uint(s1);
-        mx = fmaxf(mx, fmaxf(s0, s1));
-      }
+      for (int c = 0; c < 32; ++c) mx = fmaxf(mx, fmaxf(__uint_as_float(v0[c]), __uint_as_float(v1[c])));
+      mx *= sc;   // the scale is positive: max and scaling commute
       if (last_row && probs) {   // the logits of the visual positions; normalised once the row is complete
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
           const int ja = j0 + c - p.sys_len, jb = ja + 32;
-          if (ja >= 0 && ja < p.num_visual) probs[ja] = __uint_as_float(v0[c]);
-          if (jb >= 0 && jb < p.num_visual) probs[jb] = __uint_as_float(v1[c]);
+          if (ja >= 0 && ja < p.num_visual) probs[ja] = __uint_as_float(v0[c]) * sc;
+          if (jb >= 0 && jb < p.num_visual) probs[jb] = __uint_as_float(v1[c]) * sc;
         }
       }
       // lazy rescale: move the reference only when the maximum has run away from it
@@ -239,42 +275,48 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
         factor = ref > -INFINITY ? fast_exp2(ref - mx) : 0.f;
         ref = mx;
       }
-      if (kt > 0 && __any_sync(0xffffffffu, factor != 1.f)) {
-        // the previous P V has completed (bar_o was waited below), so O is stable: scale this row in place
-#pragma unroll 1
-        for (int cb = 0; cb < 4; ++cb) {
-          uint32_t o[32];
-          tmem_ld32(tmem_O + lane_addr + cb * 32, o);
-#pragma unroll
-          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * factor);
-          tmem_st32(tmem_O + lane_addr + cb * 32, o);
-        }
-      }
       l *= factor;
-      // probabilities, as bf16, into the swizzled A-operand tile: 8 chunks of 8 keys
-      const float rf = ref > -INFINITY ? ref : 0.f;   // a row with no key yet (padding rows) yields zeros
+      // probabilities exp2(s * sc - ref) as packed bf16 pairs (exp2(-inf) = 0 for masked keys)
+      const float nrf = ref > -INFINITY ? -ref : 0.f;   // a row with no key yet (padding rows) yields zeros
       float add = 0.f;
+      uint32_t w[32];
 #pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        uint32_t w[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int c = (ch & 3) * 8 + e * 2;
-          const float sa = __uint_as_float(ch < 4 ? v0[c] : v1[c]), sb = __uint_as_float(ch < 4 ? v0[c + 1] : v1[c + 1]);
-          const float pa = fast_exp2(sa - rf), pb = fast_exp2(sb - rf);   // exp2(-inf) = 0 for masked keys
-          add += pa + pb;
-          const __nv_bfloat162 b2 = __floats2bfloat162_rn(pa, pb);
-          w[e] = *reinterpret_cast<const uint32_t*>(&b2);
-        }
-        unsigned char* dst = sP + (r >> 3) * 1024 + (r & 7) * 128 + ((ch ^ (r & 7)) << 4);
-        *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+      for (int c = 0; c < 32; c += 2) {
+        const float pa = fast_exp2(fmaf(__uint_as_float(v0[c]), sc, nrf)), pb = fast_exp2(fmaf(__uint_as_float(v0[c + 1]), sc, nrf));
+        const float pc = fast_exp2(fmaf(__uint_as_float(v1[c]), sc, nrf)), pd = fast_exp2(fmaf(__uint_as_float(v1[c + 1]), sc, nrf));
+        add += (pa + pb) + (pc + pd);
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(pa, pb), hi = __floats2bfloat162_rn(pc, pd);
+        w[c >> 1] = *reinterpret_cast<const uint32_t*>(&lo);
+        w[16 + (c >> 1)] = *reinterpret_cast<const uint32_t*>(&hi);
       }
       l += add;
+      // P V(kt-1) must be complete before O is rescaled or P overwritten
+      if (kt > 0) {
+        ok = pf_wait(&bar_o, (kt - 1) & 1) && !*fail;
+        if (!ok) break;
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, factor != 1.f)) {
+#pragma unroll 1
+          for (int cb = 0; cb < 4; ++cb) {
+            uint32_t o[32];
+            tmem_ld32(tmem_O + lane_addr + cb * 32, o);
+#pragma unroll
+            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * factor);
+            tmem_st32(tmem_O + lane_addr + cb * 32, o);
+          }
+        }
+      }
+      // into the swizzled A-operand tile: 8 chunks of 8 keys
+#pragma unroll
+      for (int ch = 0; ch < 8; ++ch) {
+        unsigned char* dst = sP + (r >> 3) * 1024 + (r & 7) * 128 + ((ch ^ (r & 7)) << 4);
+        *reinterpret_cast<uint4*>(dst) = make_uint4(w[ch * 4], w[ch * 4 + 1], w[ch * 4 + 2], w[ch * 4 + 3]);
+      }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core
       tc_fence_before();
-      mbar_arrive_cta(&bar_read);
-      ok = pf_wait(&bar_o, ph_o) && !*fail; ph_o ^= 1;               // P V done: P may be overwritten, O is stable
+      mbar_arrive_cta(&bar_p);
     }
+    if (ok) { ok = pf_wait(&bar_o, (nkt - 1) & 1) && !*fail; }   // the last P V: O is complete
     const float inv_l = l > 0.f ? 1.f / l : 0.f;
     if (probs && (T - 1) / kTile == qt) {   // this block holds the last query row (same answer in every thread)
       // alpha of this head: exp2(logit - ref) / sum over the visual positions, with the last row's final
@@ -370,7 +412,7 @@ extern "C" st3_status st3_prefill_attend(const void* q, const void* k, const voi
       !make_map(encode, &mv, v, rows, kKeys))
     return ST3_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const int smem = kTileBytes2 + kPBytes + 2 * kKTileBytes + 1024;   // Q, P, K, V (+ alignment slack)
+  const int smem = kTileBytes2 + kPBytes + 3 * kKTileBytes + 1024;   // Q, P, V, two K buffers (+ alignment slack)
   if (cudaFuncSetAttribute(st3_prefill_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
     return ST3_ERR_CUDA;
   PrefillParams p;

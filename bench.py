@@ -346,14 +346,14 @@ def oracle_sample(wl, g, K, V, q0, q, kn, vn, nsteps, warm_steps, reps=1):
     return wl.batch * nsteps / secs, secs, threads, first, t - 1
 
 
-def prefill_attend_leg(wl, device, iters=10):
+def prefill_attend_leg(wl, device, iters=10, max_instances=2048):
     """Causal prompt attention (the step before the hot path) on the tensor cores: every layer's
     (sequence, head) instances of the workload in one call, full prompt length."""
     from paper_2412_20105_b200 import binding as B
     if wl.dtype != "bf16" or wl.head_dim != 128:
         return None
     T = wl.sys_len + wl.num_visual + wl.text_len_max
-    n = min(wl.num_layers * wl.batch * wl.num_heads, 2048)
+    n = max(wl.num_heads, min(wl.num_layers * wl.batch * wl.num_heads, max_instances))
     n -= n % wl.num_heads
     g = torch.Generator().manual_seed(wl.seed)
     mk = lambda: torch.randn(n, T, 128, generator=g).to(torch.bfloat16).to(device)
@@ -389,6 +389,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows-per-chunk", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="skip the e2e, unpruned and cpu_baseline legs")
+    ap.add_argument("--leg", default="", choices=["", "prefill_attend"],
+                    help="run one auxiliary leg alone and print its JSON (for timing or profiling that kernel)")
+    ap.add_argument("--instances", type=int, default=2048, help="cap on the (sequence, head) instances of --leg")
     args = ap.parse_args()
     wl = get_workload(args.workload)
     rank = int(os.environ.get("RANK", "0"))
@@ -434,6 +437,11 @@ def main():
     dist = world > 1
     torch.cuda.set_device(local)
     device = torch.device(f"cuda:{local}")
+    if args.leg == "prefill_attend":
+        if rank == 0:
+            print(json.dumps({"leg": args.leg, "workload": wl.name,
+                              **(prefill_attend_leg(wl, device, max(1, args.steps), args.instances) or {})}))
+        return
     if dist:
         torch.distributed.init_process_group("nccl", device_id=device)
     wl = replica_workload(wl, rank, world)

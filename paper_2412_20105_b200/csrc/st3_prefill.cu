@@ -82,6 +82,25 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "memory");
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+// 64 consecutive columns of this thread's lane in one instruction (one round trip instead of two)
+__device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x64.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, "
+      "%32, %33, %34, %35, %36, %37, %38, %39, %40, %41, %42, %43, %44, %45, %46, %47, "
+      "%48, %49, %50, %51, %52, %53, %54, %55, %56, %57, %58, %59, %60, %61, %62, %63}, [%64];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31]), "=r"(r[32]),
+        "=r"(r[33]), "=r"(r[34]), "=r"(r[35]), "=r"(r[36]), "=r"(r[37]), "=r"(r[38]), "=r"(r[39]), "=r"(r[40]),
+        "=r"(r[41]), "=r"(r[42]), "=r"(r[43]), "=r"(r[44]), "=r"(r[45]), "=r"(r[46]), "=r"(r[47]), "=r"(r[48]),
+        "=r"(r[49]), "=r"(r[50]), "=r"(r[51]), "=r"(r[52]), "=r"(r[53]), "=r"(r[54]), "=r"(r[55]), "=r"(r[56]),
+        "=r"(r[57]), "=r"(r[58]), "=r"(r[59]), "=r"(r[60]), "=r"(r[61]), "=r"(r[62]), "=r"(r[63])
+      : "r"(taddr)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -101,6 +120,15 @@ constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4
 constexpr uint32_t kIdescS = kIdescBase | ((kKeys >> 3) << 17);                 // N = 64 keys, A and B K-major
 constexpr uint32_t kIdescPV = kIdescBase | ((128u >> 3) << 17) | (1u << 16);    // N = 128 dims, B (= V) MN-major
 
+struct PfShared {   // after the tiles in dynamic shared memory
+  uint64_t bar_q, bar_k[2], bar_v[2], bar_s[2], bar_p, bar_o;
+  uint32_t tmem;
+  int fail;
+  float last[2];
+};
+constexpr int kPfSmem = kTileBytes2 + kPBytes + 4 * kKTileBytes + 128;   // Q, P, two V and two K buffers, PfShared
+static_assert(sizeof(PfShared) <= 128, "PfShared must fit its slot");
+
 struct PrefillParams {
   __nv_bfloat16* out;   // [num_inst][T][128]
   float* head_probs;    // [num_inst][num_visual] last-row probabilities per head
@@ -111,17 +139,25 @@ struct PrefillParams {
 __global__ void __launch_bounds__(kPfThreads, 2)
 st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                           const __grid_constant__ CUtensorMap map_v, const PrefillParams p) {
-  extern __shared__ __align__(1024) unsigned char smem_raw[];
-  // the dynamic window is only 16-byte aligned by contract: round up to the 1024 bytes the swizzle needs
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // Two blocks per SM leave each 113 KB: the tiles take 112 KB of it, so there is no room for alignment slack.
+  // The kernel has no static shared memory, which puts the dynamic window at the (1024-byte aligned) start of
+  // the block's allocation; the tiles come first and the small variables after them.  A misaligned window is
+  // reported, not used (the 128-byte swizzle of TMA and of the MMA descriptors assumes 1024-byte aligned tiles).
+  extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* sQ = smem;
   unsigned char* sP = sQ + kTileBytes2;
-  unsigned char* sV = sP + kPBytes;
-  unsigned char* sK2 = sV + kKTileBytes;   // two K buffers: tile t+2 replaces tile t as soon as S(t) is complete
-  __shared__ __align__(8) uint64_t bar_q, bar_k[2], bar_v, bar_s[2], bar_p, bar_o;
-  __shared__ uint32_t s_tmem;
-  __shared__ int s_fail;
-  __shared__ float s_last[2];
+  unsigned char* sV2 = sP + kPBytes;          // two V buffers: tile t+2 replaces tile t once P V(t) is complete
+  unsigned char* sK2 = sV2 + 2 * kKTileBytes; // two K buffers: tile t+2 replaces tile t once S(t) is complete
+  PfShared& sh = *reinterpret_cast<PfShared*>(sK2 + 2 * kKTileBytes);
+  uint64_t &bar_q = sh.bar_q, &bar_p = sh.bar_p, &bar_o = sh.bar_o;
+  uint64_t (&bar_k)[2] = sh.bar_k, (&bar_v)[2] = sh.bar_v, (&bar_s)[2] = sh.bar_s;
+  uint32_t& s_tmem = sh.tmem;
+  int& s_fail = sh.fail;
+  float (&s_last)[2] = sh.last;
+  if (smem_u32(smem) & 1023u) {
+    if (threadIdx.x == 0 && p.status) atomicOr(p.status, ST3_DEV_RANGE);
+    return;
+  }
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int qt = blockIdx.x, inst = blockIdx.y;
@@ -130,7 +166,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   const int nkt = (min(T, (qt + 1) * kTile) + kKeys - 1) / kKeys;  // causal: key tiles up to the diagonal
 
   if (tid == 0) {
-    mbar_init(&bar_q, 1); mbar_init(&bar_k[0], 1); mbar_init(&bar_k[1], 1); mbar_init(&bar_v, 1);
+    mbar_init(&bar_q, 1); mbar_init(&bar_k[0], 1); mbar_init(&bar_k[1], 1); mbar_init(&bar_v[0], 1); mbar_init(&bar_v[1], 1);
     mbar_init(&bar_s[0], 1); mbar_init(&bar_s[1], 1); mbar_init(&bar_o, 1);
     mbar_init(&bar_p, 128);
     s_fail = 0;
@@ -161,9 +197,10 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       tma_load_2d(d + kKBoxBytes, &map_k, 64, row_base + kt * kKeys, &bar_k[kt & 1]);
     };
     auto load_v = [&](int kt) {
-      mbar_expect_tx(&bar_v, kKTileBytes);
-      tma_load_2d(sV, &map_v, 0, row_base + kt * kKeys, &bar_v);
-      tma_load_2d(sV + kKBoxBytes, &map_v, 64, row_base + kt * kKeys, &bar_v);
+      unsigned char* d = sV2 + (kt & 1) * kKTileBytes;
+      mbar_expect_tx(&bar_v[kt & 1], kKTileBytes);
+      tma_load_2d(d, &map_v, 0, row_base + kt * kKeys, &bar_v[kt & 1]);
+      tma_load_2d(d + kKBoxBytes, &map_v, 64, row_base + kt * kKeys, &bar_v[kt & 1]);
     };
     // S(kt) = Q K(kt)^T: 8 steps of 16 along the head dimension
     auto issue_s = [&](int kt) {
@@ -184,6 +221,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       load_k(0);
       if (nkt > 1) load_k(1);
       load_v(0);
+      if (nkt > 1) load_v(1);
     }
     ok = pf_wait(&bar_q, 0);
     // prologue: S(0) and S(1); then K(2), K(3) into the buffers they leave
@@ -203,12 +241,13 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       // P(kt) is in shared memory (its writers have also seen P V(kt-1) complete) and V(kt) has landed
       ok = pf_wait(&bar_p, kt & 1);
       if (!ok) break;
-      ok = pf_wait(&bar_v, kt & 1);
+      ok = pf_wait(&bar_v[kt & 1], (kt >> 1) & 1);
       if (!ok) break;
       if (kt + 2 < nkt) { ok = pf_wait(&bar_k[kt & 1], ((kt + 2) >> 1) & 1); if (!ok) break; }
       tc_fence_after();
       if (lane == 0) {
         // O += P V: 4 steps of 16 keys; V is the MN-major operand (two 64-dim boxes 8 KB apart)
+        const unsigned char* sV = sV2 + (kt & 1) * kKTileBytes;
 #pragma unroll
         for (int ks = 0; ks < kKeys / 16; ++ks)
           umma_bf16(tmem_O, smem_desc(smem_u32(sP) + ks * 32, 16), smem_desc(smem_u32(sV) + ks * 2048, kKBoxBytes),
@@ -220,7 +259,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       // refill what these MMAs release: V's buffer after P V(kt), K's buffer after S(kt+2)
       ok = pf_wait(&bar_o, kt & 1);
       if (!ok) break;
-      if (lane == 0 && kt + 1 < nkt) load_v(kt + 1);
+      if (lane == 0 && kt + 2 < nkt) load_v(kt + 2);
       if (kt + 4 < nkt) {
         ok = pf_wait(&bar_s[kt & 1], ((kt + 2) >> 1) & 1);
         if (!ok) break;
@@ -246,27 +285,25 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       if (!ok) break;
       tc_fence_after();
       const uint32_t tmem_S = tmem + (uint32_t)(kt & 1) * kKeys;
-      uint32_t v0[32], v1[32];
-      tmem_ld32(tmem_S + lane_addr, v0);
-      tmem_ld32(tmem_S + lane_addr + 32, v1);
+      uint32_t v[64];
+      tmem_ld64(tmem_S + lane_addr, v);
       const int j0 = kt * kKeys;
       if (j0 + kKeys > qt * kTile + 1 || j0 + kKeys > T) {   // the tile touches the diagonal or the end of the prompt
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          if (!(live && j0 + c <= qi && j0 + c < T)) v0[c] = 0xff800000u;
-          if (!(live && j0 + 32 + c <= qi && j0 + 32 + c < T)) v1[c] = 0xff800000u;
-        }
+        for (int c = 0; c < 64; ++c)
+          if (!(live && j0 + c <= qi && j0 + c < T)) v[c] = 0xff800000u;
       }
-      float mx = -INFINITY;
+      float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int c = 0; c < 32; ++c) mx = fmaxf(mx, fmaxf(__uint_as_float(v0[c]), __uint_as_float(v1[c])));
-      mx *= sc;   // the scale is positive: max and scaling commute
+      for (int c = 0; c < 64; c += 8)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) m4[e] = fmaxf(m4[e], fmaxf(__uint_as_float(v[c + e]), __uint_as_float(v[c + 4 + e])));
+      const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * sc;   // the scale is positive: max and scaling commute
       if (last_row && probs) {   // the logits of the visual positions; normalised once the row is complete
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          const int ja = j0 + c - p.sys_len, jb = ja + 32;
-          if (ja >= 0 && ja < p.num_visual) probs[ja] = __uint_as_float(v0[c]) * sc;
-          if (jb >= 0 && jb < p.num_visual) probs[jb] = __uint_as_float(v1[c]) * sc;
+        for (int c = 0; c < 64; ++c) {
+          const int ja = j0 + c - p.sys_len;
+          if (ja >= 0 && ja < p.num_visual) probs[ja] = __uint_as_float(v[c]) * sc;
         }
       }
       // lazy rescale: move the reference only when the maximum has run away from it
@@ -276,20 +313,24 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
         ref = mx;
       }
       l *= factor;
-      // probabilities exp2(s * sc - ref) as packed bf16 pairs (exp2(-inf) = 0 for masked keys)
+      // probabilities exp2(s * sc - ref) as packed bf16 pairs (exp2(-inf) = 0 for masked keys); the scaling runs
+      // as packed two-wide FMAs
       const float nrf = ref > -INFINITY ? -ref : 0.f;   // a row with no key yet (padding rows) yields zeros
-      float add = 0.f;
+      const u64 sc2 = pack2(sc, sc), nrf2 = pack2(nrf, nrf);
+      float add[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t w[32];
 #pragma unroll
-      for (int c = 0; c < 32; c += 2) {
-        const float pa = fast_exp2(fmaf(__uint_as_float(v0[c]), sc, nrf)), pb = fast_exp2(fmaf(__uint_as_float(v0[c + 1]), sc, nrf));
-        const float pc = fast_exp2(fmaf(__uint_as_float(v1[c]), sc, nrf)), pd = fast_exp2(fmaf(__uint_as_float(v1[c + 1]), sc, nrf));
-        add += (pa + pb) + (pc + pd);
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(pa, pb), hi = __floats2bfloat162_rn(pc, pd);
-        w[c >> 1] = *reinterpret_cast<const uint32_t*>(&lo);
-        w[16 + (c >> 1)] = *reinterpret_cast<const uint32_t*>(&hi);
+      for (int c = 0; c < 64; c += 2) {
+        u64 t2 = nrf2;
+        fma2(t2, pack2(__uint_as_float(v[c]), __uint_as_float(v[c + 1])), sc2);
+        float ta, tb;
+        split2(t2, ta, tb);
+        const float pa = fast_exp2(ta), pb = fast_exp2(tb);
+        add[(c >> 1) & 3] += pa + pb;
+        const __nv_bfloat162 b2 = __floats2bfloat162_rn(pa, pb);
+        w[c >> 1] = *reinterpret_cast<const uint32_t*>(&b2);
       }
-      l += add;
+      l += (add[0] + add[1]) + (add[2] + add[3]);
       // P V(kt-1) must be complete before O is rescaled or P overwritten
       if (kt > 0) {
         ok = pf_wait(&bar_o, (kt - 1) & 1) && !*fail;
@@ -412,7 +453,7 @@ extern "C" st3_status st3_prefill_attend(const void* q, const void* k, const voi
       !make_map(encode, &mv, v, rows, kKeys))
     return ST3_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  const int smem = kTileBytes2 + kPBytes + 3 * kKTileBytes + 1024;   // Q, P, V, two K buffers (+ alignment slack)
+  const int smem = kPfSmem;
   if (cudaFuncSetAttribute(st3_prefill_attend_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
     return ST3_ERR_CUDA;
   PrefillParams p;

@@ -115,6 +115,38 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+__device__ __forceinline__ u64 add2(u64 a, u64 b) {
+  u64 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ u64 fma2r(u64 a, u64 b, u64 c) {
+  u64 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+// exp2 of a pair on the FMA pipe, for arguments <= 8 or so: the special-function unit, at a quarter of the FMA
+// rate, is what bounds the softmax, so half of the exponentials are computed here instead.  x is clamped to
+// >= -120, split as j + f with j = round(x) (adding and subtracting 1.5 * 2^23) and f in [-0.5, 0.5]; 2^f is a
+// cubic (relative error 7.5e-5, below the bf16 rounding of P); j is added into the exponent field.
+__device__ __forceinline__ void exp2_pair_fma(u64 x2, float& pa, float& pb) {
+  float xa, xb;
+  split2(x2, xa, xb);
+  x2 = pack2(fmaxf(xa, -120.f), fmaxf(xb, -120.f));
+  const u64 magic = pack2(12582912.f, 12582912.f);
+  const u64 t2 = add2(x2, magic);
+  const u64 nj = fma2r(t2, pack2(-1.f, -1.f), magic);   // -(round(x))
+  const u64 f2 = add2(x2, nj);
+  u64 r2 = fma2r(pack2(0.05517132f, 0.05517132f), f2, pack2(0.24261054f, 0.24261054f));
+  r2 = fma2r(r2, f2, pack2(0.69326097f, 0.69326097f));
+  r2 = fma2r(r2, f2, pack2(0.99992812f, 0.99992812f));
+  float ra, rb, ta, tb;
+  split2(r2, ra, rb);
+  split2(t2, ta, tb);
+  pa = __uint_as_float(__float_as_uint(ra) + (__float_as_uint(ta) << 23));
+  pb = __uint_as_float(__float_as_uint(rb) + (__float_as_uint(tb) << 23));
+}
+
 // kind::f16 instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128.
 constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescS = kIdescBase | ((kKeys >> 3) << 17);                 // N = 64 keys, A and B K-major
@@ -281,7 +313,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     float* probs = p.head_probs ? p.head_probs + (size_t)inst * p.num_visual : nullptr;
     const bool last_row = live && qi == T - 1;
     for (int kt = 0; kt < nkt && ok; ++kt) {
-      ok = pf_wait(&bar_s[kt & 1], (kt >> 1) & 1) && !*fail;
+      ok = pf_wait(&bar_s[kt & 1], (kt >> 1) & 1);   // a failed control warp stops issuing: this wait then runs out
       if (!ok) break;
       tc_fence_after();
       const uint32_t tmem_S = tmem + (uint32_t)(kt & 1) * kKeys;
@@ -299,11 +331,20 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
 #pragma unroll
         for (int e = 0; e < 4; ++e) m4[e] = fmaxf(m4[e], fmaxf(__uint_as_float(v[c + e]), __uint_as_float(v[c + 4 + e])));
       const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * sc;   // the scale is positive: max and scaling commute
-      if (last_row && probs) {   // the logits of the visual positions; normalised once the row is complete
+      if (probs && (T - 1) / kTile == qt && ((T - 1) % kTile) >> 5 == warp) {
+        // the last query row lives in one lane of this warp: hand its logits on the visual positions to the
+        // whole warp, which stores them coalesced; they are normalised once the row is complete
+        const int src = (T - 1) & 31;
 #pragma unroll
-        for (int c = 0; c < 64; ++c) {
-          const int ja = j0 + c - p.sys_len;
-          if (ja >= 0 && ja < p.num_visual) probs[ja] = __uint_as_float(v[c]) * sc;
+        for (int c = 0; c < 64; c += 32) {
+          float mine = 0.f;
+#pragma unroll
+          for (int e = 0; e < 32; ++e) {
+            const float x = __shfl_sync(0xffffffffu, __uint_as_float(v[c + e]), src);
+            if (lane == e) mine = x;
+          }
+          const int ja = j0 + c + lane - p.sys_len;
+          if (ja >= 0 && ja < p.num_visual) probs[ja] = mine * sc;
         }
       }
       // lazy rescale: move the reference only when the maximum has run away from it
@@ -323,9 +364,14 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       for (int c = 0; c < 64; c += 2) {
         u64 t2 = nrf2;
         fma2(t2, pack2(__uint_as_float(v[c]), __uint_as_float(v[c + 1])), sc2);
-        float ta, tb;
-        split2(t2, ta, tb);
-        const float pa = fast_exp2(ta), pb = fast_exp2(tb);
+        float pa, pb;
+        if ((c >> 1) & 1) {
+          exp2_pair_fma(t2, pa, pb);
+        } else {
+          float ta, tb;
+          split2(t2, ta, tb);
+          pa = fast_exp2(ta); pb = fast_exp2(tb);
+        }
         add[(c >> 1) & 3] += pa + pb;
         const __nv_bfloat162 b2 = __floats2bfloat162_rn(pa, pb);
         w[c >> 1] = *reinterpret_cast<const uint32_t*>(&b2);
@@ -333,7 +379,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       l += (add[0] + add[1]) + (add[2] + add[3]);
       // P V(kt-1) must be complete before O is rescaled or P overwritten
       if (kt > 0) {
-        ok = pf_wait(&bar_o, (kt - 1) & 1) && !*fail;
+        ok = pf_wait(&bar_o, (kt - 1) & 1);
         if (!ok) break;
         tc_fence_after();
         if (__any_sync(0xffffffffu, factor != 1.f)) {

@@ -29,7 +29,6 @@ constexpr int kBoxBytes = 128 * 128;  // one TMA box of Q: 128 rows x 64 bf16
 constexpr int kTileBytes2 = 2 * kBoxBytes;
 constexpr int kKBoxBytes = kKeys * 128;  // one TMA box of K or V: 64 rows x 64 bf16
 constexpr int kKTileBytes = 2 * kKBoxBytes;
-constexpr int kPBytes = kTile * kKeys * 2;  // probabilities of one tile, bf16
 constexpr uint32_t kTmemCols = 256;   // S in columns [0,64), O in [128,256)
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -64,6 +63,17 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
       :
       : "r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "memory");
+}
+// the same with the A operand in tensor memory (lane = row, two bf16 per 32-bit column along K)
+__device__ __forceinline__ void umma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      :
+      : "r"(tmem_d), "r"(tmem_a), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
@@ -158,7 +168,7 @@ struct PfShared {   // after the tiles in dynamic shared memory
   int fail;
   float last[2];
 };
-constexpr int kPfSmem = kTileBytes2 + kPBytes + 4 * kKTileBytes + 128;   // Q, P, two V and two K buffers, PfShared
+constexpr int kPfSmem = kTileBytes2 + 4 * kKTileBytes + 128;   // Q, two V and two K buffers, PfShared
 static_assert(sizeof(PfShared) <= 128, "PfShared must fit its slot");
 
 struct PrefillParams {
@@ -177,8 +187,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   // reported, not used (the 128-byte swizzle of TMA and of the MMA descriptors assumes 1024-byte aligned tiles).
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* sQ = smem;
-  unsigned char* sP = sQ + kTileBytes2;
-  unsigned char* sV2 = sP + kPBytes;          // two V buffers: tile t+2 replaces tile t once P V(t) is complete
+  unsigned char* sV2 = sQ + kTileBytes2;      // two V buffers: tile t+2 replaces tile t once P V(t) is complete
   unsigned char* sK2 = sV2 + 2 * kKTileBytes; // two K buffers: tile t+2 replaces tile t once S(t) is complete
   PfShared& sh = *reinterpret_cast<PfShared*>(sK2 + 2 * kKTileBytes);
   uint64_t &bar_q = sh.bar_q, &bar_p = sh.bar_p, &bar_o = sh.bar_o;
@@ -278,12 +287,14 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       if (kt + 2 < nkt) { ok = pf_wait(&bar_k[kt & 1], ((kt + 2) >> 1) & 1); if (!ok) break; }
       tc_fence_after();
       if (lane == 0) {
-        // O += P V: 4 steps of 16 keys; V is the MN-major operand (two 64-dim boxes 8 KB apart)
+        // O += P V: 4 steps of 16 keys; P is read from tensor memory, where it replaced the first half of its
+        // S tile (8 columns per 16 keys); V is the MN-major operand (two 64-dim boxes 8 KB apart)
         const unsigned char* sV = sV2 + (kt & 1) * kKTileBytes;
+        const uint32_t tmem_P = tmem + (uint32_t)(kt & 1) * kKeys;
 #pragma unroll
         for (int ks = 0; ks < kKeys / 16; ++ks)
-          umma_bf16(tmem_O, smem_desc(smem_u32(sP) + ks * 32, 16), smem_desc(smem_u32(sV) + ks * 2048, kKBoxBytes),
-                    kIdescPV, (kt > 0 || ks > 0));
+          umma_bf16_ta(tmem_O, tmem_P + ks * 8, smem_desc(smem_u32(sV) + ks * 2048, kKBoxBytes), kIdescPV,
+                       (kt > 0 || ks > 0));
         umma_commit(&bar_o);
         if (kt + 2 < nkt) issue_s(kt + 2);   // into the S buffer whose tile the softmax warps have just left
       }
@@ -377,7 +388,9 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
         w[c >> 1] = *reinterpret_cast<const uint32_t*>(&b2);
       }
       l += (add[0] + add[1]) + (add[2] + add[3]);
-      // P V(kt-1) must be complete before O is rescaled or P overwritten
+      // P V(kt-1) must be complete before O is rescaled in place.  Every thread waits for it at every step, needed
+      // or not: that keeps a fast thread from arriving for tile kt+1 while a slow one still owes its arrival
+      // for tile kt, and keeps every waiter on this barrier's current phase.
       if (kt > 0) {
         ok = pf_wait(&bar_o, (kt - 1) & 1);
         if (!ok) break;
@@ -393,13 +406,9 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
           }
         }
       }
-      // into the swizzled A-operand tile: 8 chunks of 8 keys
-#pragma unroll
-      for (int ch = 0; ch < 8; ++ch) {
-        unsigned char* dst = sP + (r >> 3) * 1024 + (r & 7) * 128 + ((ch ^ (r & 7)) << 4);
-        *reinterpret_cast<uint4*>(dst) = make_uint4(w[ch * 4], w[ch * 4 + 1], w[ch * 4 + 2], w[ch * 4 + 3]);
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // P is read by the tensor core
+      // P replaces the first 32 columns of this S tile (only this thread reads or writes this lane of it, and
+      // S(kt+2) lands there after P V(kt) in the tensor pipe's order)
+      tmem_st32(tmem_S + lane_addr, w);
       tc_fence_before();
       mbar_arrive_cta(&bar_p);
     }

@@ -50,30 +50,42 @@ __device__ __forceinline__ bool pf_wait(uint64_t* bar, uint32_t parity) {
   }
   return true;
 }
-// Shared-memory matrix descriptor: 128-byte swizzle, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes) {
-  return (uint64_t)((addr >> 4) & 0x3fffu) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) |
-         (1ull << 46) | (2ull << 61);
+// The whole warp waits and takes the same verdict: the tensor-memory accesses and __syncwarp that follow a wait
+// are warp-wide, so a timeout must not split the warp.
+__device__ __forceinline__ bool pf_wait_warp(uint64_t* bar, uint32_t parity) {
+  return __all_sync(0xffffffffu, pf_wait(bar, parity));
 }
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
+// Shared-memory matrix descriptors: 128-byte swizzle, 8-row groups 1024 bytes apart.
+// The descriptor's high word is the same for every operand here; the low word is the address field plus the
+// leading-dimension byte offset, so stepping through a tile is one 32-bit add (shared addresses stay below
+// 2^18, i.e. inside the 14-bit field, whatever is added).
+constexpr uint32_t kDescHi = (uint32_t)(1024 >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+  return ((addr >> 4) & 0x3fffu) | ((lbo_bytes >> 4) << 16);
+}
+// One MMA step (K = 16): D[tmem_d] (+)= A * B with both operands in shared memory.  `accumulate` is a
+// compile-time constant or a value fixed for the tile at every call site.
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %6};\n\t"
+      "mov.b64 db, {%2, %6};\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, {%5, %5, %5, %5}, p;\n\t}"
       :
-      : "r"(tmem_d), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "r"(tmem_d), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(0u), "r"(kDescHi)
       : "memory");
 }
 // the same with the A operand in tensor memory (lane = row, two bf16 per 32-bit column along K)
-__device__ __forceinline__ void umma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, uint64_t b_desc, uint32_t idesc,
+__device__ __forceinline__ void umma_bf16_ta(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t idesc,
                                              uint32_t accumulate) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\t"
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %6};\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %5, %5, %5}, p;\n\t}"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, {%5, %5, %5, %5}, p;\n\t}"
       :
-      : "r"(tmem_d), "r"(tmem_a), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u)
+      : "r"(tmem_d), "r"(tmem_a), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(0u), "r"(kDescHi)
       : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
@@ -244,14 +256,16 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       tma_load_2d(d + kKBoxBytes, &map_v, 64, row_base + kt * kKeys, &bar_v[kt & 1]);
     };
     // S(kt) = Q K(kt)^T: 8 steps of 16 along the head dimension
+    const uint32_t q_lo = desc_lo(smem_u32(sQ), 16), k_lo = desc_lo(smem_u32(sK2), 16);
+    const uint32_t v_lo = desc_lo(smem_u32(sV2), kKBoxBytes);
     auto issue_s = [&](int kt) {
-      const unsigned char* sK = sK2 + (kt & 1) * kKTileBytes;
+      const uint32_t kb = k_lo + (uint32_t)(kt & 1) * (kKTileBytes >> 4);
       const uint32_t tmem_S = tmem + (uint32_t)(kt & 1) * kKeys;
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         const uint32_t offq = (ks >> 2) * kBoxBytes + (ks & 3) * 32;
         const uint32_t offk = (ks >> 2) * kKBoxBytes + (ks & 3) * 32;
-        umma_bf16(tmem_S, smem_desc(smem_u32(sQ) + offq, 16), smem_desc(smem_u32(sK) + offk, 16), kIdescS, ks > 0);
+        umma_bf16(tmem_S, q_lo + (offq >> 4), kb + (offk >> 4), kIdescS, ks > 0);
       }
       umma_commit(&bar_s[kt & 1]);
     };
@@ -264,47 +278,46 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       load_v(0);
       if (nkt > 1) load_v(1);
     }
-    ok = pf_wait(&bar_q, 0);
+    ok = pf_wait_warp(&bar_q, 0);
     // prologue: S(0) and S(1); then K(2), K(3) into the buffers they leave
     for (int kt = 0; kt < 2 && kt < nkt && ok; ++kt) {
-      ok = pf_wait(&bar_k[kt], 0);
+      ok = pf_wait_warp(&bar_k[kt], 0);
       if (!ok) break;
       tc_fence_after();
       if (lane == 0) issue_s(kt);
       __syncwarp();
     }
     for (int kt = 0; kt < 2 && kt + 2 < nkt && ok; ++kt) {
-      ok = pf_wait(&bar_s[kt], 0);
+      ok = pf_wait_warp(&bar_s[kt], 0);
       if (ok && lane == 0) load_k(kt + 2);
       __syncwarp();
     }
     for (int kt = 0; kt < nkt && ok; ++kt) {
       // P(kt) is in shared memory (its writers have also seen P V(kt-1) complete) and V(kt) has landed
-      ok = pf_wait(&bar_p, kt & 1);
+      ok = pf_wait_warp(&bar_p, kt & 1);
       if (!ok) break;
-      ok = pf_wait(&bar_v[kt & 1], (kt >> 1) & 1);
+      ok = pf_wait_warp(&bar_v[kt & 1], (kt >> 1) & 1);
       if (!ok) break;
-      if (kt + 2 < nkt) { ok = pf_wait(&bar_k[kt & 1], ((kt + 2) >> 1) & 1); if (!ok) break; }
+      if (kt + 2 < nkt) { ok = pf_wait_warp(&bar_k[kt & 1], ((kt + 2) >> 1) & 1); if (!ok) break; }
       tc_fence_after();
       if (lane == 0) {
         // O += P V: 4 steps of 16 keys; P is read from tensor memory, where it replaced the first half of its
         // S tile (8 columns per 16 keys); V is the MN-major operand (two 64-dim boxes 8 KB apart)
-        const unsigned char* sV = sV2 + (kt & 1) * kKTileBytes;
+        const uint32_t vb = v_lo + (uint32_t)(kt & 1) * (kKTileBytes >> 4);
         const uint32_t tmem_P = tmem + (uint32_t)(kt & 1) * kKeys;
 #pragma unroll
         for (int ks = 0; ks < kKeys / 16; ++ks)
-          umma_bf16_ta(tmem_O, tmem_P + ks * 8, smem_desc(smem_u32(sV) + ks * 2048, kKBoxBytes), kIdescPV,
-                       (kt > 0 || ks > 0));
+          umma_bf16_ta(tmem_O, tmem_P + ks * 8, vb + ks * (2048 >> 4), kIdescPV, (kt > 0 || ks > 0));
         umma_commit(&bar_o);
         if (kt + 2 < nkt) issue_s(kt + 2);   // into the S buffer whose tile the softmax warps have just left
       }
       __syncwarp();
       // refill what these MMAs release: V's buffer after P V(kt), K's buffer after S(kt+2)
-      ok = pf_wait(&bar_o, kt & 1);
+      ok = pf_wait_warp(&bar_o, kt & 1);
       if (!ok) break;
       if (lane == 0 && kt + 2 < nkt) load_v(kt + 2);
       if (kt + 4 < nkt) {
-        ok = pf_wait(&bar_s[kt & 1], ((kt + 2) >> 1) & 1);
+        ok = pf_wait_warp(&bar_s[kt & 1], ((kt + 2) >> 1) & 1);
         if (!ok) break;
         if (lane == 0) load_k(kt + 4);
       }
@@ -324,7 +337,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     float* probs = p.head_probs ? p.head_probs + (size_t)inst * p.num_visual : nullptr;
     const bool last_row = live && qi == T - 1;
     for (int kt = 0; kt < nkt && ok; ++kt) {
-      ok = pf_wait(&bar_s[kt & 1], (kt >> 1) & 1);   // a failed control warp stops issuing: this wait then runs out
+      ok = pf_wait_warp(&bar_s[kt & 1], (kt >> 1) & 1);   // a failed control warp stops issuing: this wait then runs out
       if (!ok) break;
       tc_fence_after();
       const uint32_t tmem_S = tmem + (uint32_t)(kt & 1) * kKeys;
@@ -392,7 +405,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       // or not: that keeps a fast thread from arriving for tile kt+1 while a slow one still owes its arrival
       // for tile kt, and keeps every waiter on this barrier's current phase.
       if (kt > 0) {
-        ok = pf_wait(&bar_o, (kt - 1) & 1);
+        ok = pf_wait_warp(&bar_o, (kt - 1) & 1);
         if (!ok) break;
         tc_fence_after();
         if (__any_sync(0xffffffffu, factor != 1.f)) {
@@ -412,7 +425,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       tc_fence_before();
       mbar_arrive_cta(&bar_p);
     }
-    if (ok) { ok = pf_wait(&bar_o, (nkt - 1) & 1) && !*fail; }   // the last P V: O is complete
+    if (ok) { ok = pf_wait_warp(&bar_o, (nkt - 1) & 1) && !*fail; }   // the last P V: O is complete
     const float inv_l = l > 0.f ? 1.f / l : 0.f;
     if (probs && (T - 1) / kTile == qt) {   // this block holds the last query row (same answer in every thread)
       // alpha of this head: exp2(logit - ref) / sum over the visual positions, with the last row's final

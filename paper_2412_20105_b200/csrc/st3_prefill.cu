@@ -29,6 +29,7 @@ constexpr int kBoxBytes = 128 * 128;  // one TMA box of Q: 128 rows x 64 bf16
 constexpr int kTileBytes2 = 2 * kBoxBytes;
 constexpr int kKBoxBytes = kKeys * 128;  // one TMA box of K or V: 64 rows x 64 bf16
 constexpr int kKTileBytes = 2 * kKBoxBytes;
+constexpr int kPolyPhase = 3;         // pairs (of every four) whose exponentials run on the FMA pipe; 4 = none
 constexpr uint32_t kTmemCols = 256;   // S in columns [0,64), O in [128,256)
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -137,6 +138,11 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
 __device__ __forceinline__ u64 add2(u64 a, u64 b) {
   u64 d;
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
@@ -353,7 +359,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
 #pragma unroll
       for (int c = 0; c < 64; c += 8)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) m4[e] = fmaxf(m4[e], fmaxf(__uint_as_float(v[c + e]), __uint_as_float(v[c + 4 + e])));
+        for (int e = 0; e < 4; ++e) m4[e] = fmax3(m4[e], __uint_as_float(v[c + e]), __uint_as_float(v[c + 4 + e]));
       const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * sc;   // the scale is positive: max and scaling commute
       if (probs && (T - 1) / kTile == qt && ((T - 1) % kTile) >> 5 == warp) {
         // the last query row lives in one lane of this warp: hand its logits on the visual positions to the
@@ -382,25 +388,25 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       // as packed two-wide FMAs
       const float nrf = ref > -INFINITY ? -ref : 0.f;   // a row with no key yet (padding rows) yields zeros
       const u64 sc2 = pack2(sc, sc), nrf2 = pack2(nrf, nrf);
-      float add[4] = {0.f, 0.f, 0.f, 0.f};
+      u64 add[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};   // row sum, as two packed pairs
       uint32_t w[32];
 #pragma unroll
       for (int c = 0; c < 64; c += 2) {
         u64 t2 = nrf2;
         fma2(t2, pack2(__uint_as_float(v[c]), __uint_as_float(v[c + 1])), sc2);
         float pa, pb;
-        if ((c >> 1) & 1) {
+        if (((c >> 1) & 3) == kPolyPhase) {
           exp2_pair_fma(t2, pa, pb);
         } else {
           float ta, tb;
           split2(t2, ta, tb);
           pa = fast_exp2(ta); pb = fast_exp2(tb);
         }
-        add[(c >> 1) & 3] += pa + pb;
+        add[(c >> 1) & 1] = add2(add[(c >> 1) & 1], pack2(pa, pb));
         const __nv_bfloat162 b2 = __floats2bfloat162_rn(pa, pb);
         w[c >> 1] = *reinterpret_cast<const uint32_t*>(&b2);
       }
-      l += (add[0] + add[1]) + (add[2] + add[3]);
+      l += sum2(add2(add[0], add[1]));
       // P V(kt-1) must be complete before O is rescaled in place.  Every thread waits for it at every step, needed
       // or not: that keeps a fast thread from arriving for tile kt+1 while a slow one still owes its arrival
       // for tile kt, and keeps every waiter on this barrier's current phase.

@@ -29,7 +29,7 @@ constexpr int kBoxBytes = 128 * 128;  // one TMA box of Q: 128 rows x 64 bf16
 constexpr int kTileBytes2 = 2 * kBoxBytes;
 constexpr int kKBoxBytes = kKeys * 128;  // one TMA box of K or V: 64 rows x 64 bf16
 constexpr int kKTileBytes = 2 * kKBoxBytes;
-constexpr int kPolyPhase = 3;         // pairs (of every four) whose exponentials run on the FMA pipe; 4 = none
+constexpr int kPolyPhase = 4;         // pairs (of every four) whose exponentials run on the FMA pipe; 4 = none
 constexpr uint32_t kTmemCols = 256;   // S in columns [0,64), O in [128,256)
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -181,12 +181,12 @@ constexpr uint32_t kIdescS = kIdescBase | ((kKeys >> 3) << 17);                 
 constexpr uint32_t kIdescPV = kIdescBase | ((128u >> 3) << 17) | (1u << 16);    // N = 128 dims, B (= V) MN-major
 
 struct PfShared {   // after the tiles in dynamic shared memory
-  uint64_t bar_q, bar_k[2], bar_v[2], bar_s[2], bar_p, bar_o;
+  uint64_t bar_q, bar_k[3], bar_v[2], bar_s[2], bar_p[2], bar_o, bar_done;
   uint32_t tmem;
   int fail;
   float last[2];
 };
-constexpr int kPfSmem = kTileBytes2 + 4 * kKTileBytes + 128;   // Q, two V and two K buffers, PfShared
+constexpr int kPfSmem = kTileBytes2 + 5 * kKTileBytes + 128;   // Q, two V and three K buffers, PfShared
 static_assert(sizeof(PfShared) <= 128, "PfShared must fit its slot");
 
 struct PrefillParams {
@@ -206,10 +206,12 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* sQ = smem;
   unsigned char* sV2 = sQ + kTileBytes2;      // two V buffers: tile t+2 replaces tile t once P V(t) is complete
-  unsigned char* sK2 = sV2 + 2 * kKTileBytes; // two K buffers: tile t+2 replaces tile t once S(t) is complete
-  PfShared& sh = *reinterpret_cast<PfShared*>(sK2 + 2 * kKTileBytes);
-  uint64_t &bar_q = sh.bar_q, &bar_p = sh.bar_p, &bar_o = sh.bar_o;
-  uint64_t (&bar_k)[2] = sh.bar_k, (&bar_v)[2] = sh.bar_v, (&bar_s)[2] = sh.bar_s;
+  unsigned char* sK2 = sV2 + 2 * kKTileBytes; // three K buffers: tile t+3 replaces tile t once S(t) is complete
+  PfShared& sh = *reinterpret_cast<PfShared*>(sK2 + 3 * kKTileBytes);
+  uint64_t &bar_q = sh.bar_q, &bar_o = sh.bar_o, &bar_done = sh.bar_done;
+  uint64_t (&bar_p)[2] = sh.bar_p;
+  uint64_t (&bar_k)[3] = sh.bar_k;
+  uint64_t (&bar_v)[2] = sh.bar_v, (&bar_s)[2] = sh.bar_s;
   uint32_t& s_tmem = sh.tmem;
   int& s_fail = sh.fail;
   float (&s_last)[2] = sh.last;
@@ -225,9 +227,9 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   const int nkt = (min(T, (qt + 1) * kTile) + kKeys - 1) / kKeys;  // causal: key tiles up to the diagonal
 
   if (tid == 0) {
-    mbar_init(&bar_q, 1); mbar_init(&bar_k[0], 1); mbar_init(&bar_k[1], 1); mbar_init(&bar_v[0], 1); mbar_init(&bar_v[1], 1);
+    mbar_init(&bar_q, 1); mbar_init(&bar_k[0], 1); mbar_init(&bar_k[1], 1); mbar_init(&bar_k[2], 1); mbar_init(&bar_v[0], 1); mbar_init(&bar_v[1], 1);
     mbar_init(&bar_s[0], 1); mbar_init(&bar_s[1], 1); mbar_init(&bar_o, 1);
-    mbar_init(&bar_p, 128);
+    mbar_init(&bar_p[0], 128); mbar_init(&bar_p[1], 128); mbar_init(&bar_done, 1);
     s_fail = 0;
     mbar_fence_init();
   }
@@ -250,10 +252,10 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     // the softmax of tile t ends, so the softmax warps never wait for the tensor cores in steady state.
     bool ok = true;
     auto load_k = [&](int kt) {
-      unsigned char* d = sK2 + (kt & 1) * kKTileBytes;
-      mbar_expect_tx(&bar_k[kt & 1], kKTileBytes);
-      tma_load_2d(d, &map_k, 0, row_base + kt * kKeys, &bar_k[kt & 1]);
-      tma_load_2d(d + kKBoxBytes, &map_k, 64, row_base + kt * kKeys, &bar_k[kt & 1]);
+      unsigned char* d = sK2 + (kt % 3) * kKTileBytes;
+      mbar_expect_tx(&bar_k[kt % 3], kKTileBytes);
+      tma_load_2d(d, &map_k, 0, row_base + kt * kKeys, &bar_k[kt % 3]);
+      tma_load_2d(d + kKBoxBytes, &map_k, 64, row_base + kt * kKeys, &bar_k[kt % 3]);
     };
     auto load_v = [&](int kt) {
       unsigned char* d = sV2 + (kt & 1) * kKTileBytes;
@@ -265,7 +267,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     const uint32_t q_lo = desc_lo(smem_u32(sQ), 16), k_lo = desc_lo(smem_u32(sK2), 16);
     const uint32_t v_lo = desc_lo(smem_u32(sV2), kKBoxBytes);
     auto issue_s = [&](int kt) {
-      const uint32_t kb = k_lo + (uint32_t)(kt & 1) * (kKTileBytes >> 4);
+      const uint32_t kb = k_lo + (uint32_t)(kt % 3) * (kKTileBytes >> 4);
       const uint32_t tmem_S = tmem + (uint32_t)(kt & 1) * kKeys;
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
@@ -281,11 +283,12 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       tma_load_2d(sQ + kBoxBytes, &map_q, 64, row_base + qt * kTile, &bar_q);
       load_k(0);
       if (nkt > 1) load_k(1);
+      if (nkt > 2) load_k(2);
       load_v(0);
       if (nkt > 1) load_v(1);
     }
     ok = pf_wait_warp(&bar_q, 0);
-    // prologue: S(0) and S(1); then K(2), K(3) into the buffers they leave
+    // prologue: S(0) and S(1)
     for (int kt = 0; kt < 2 && kt < nkt && ok; ++kt) {
       ok = pf_wait_warp(&bar_k[kt], 0);
       if (!ok) break;
@@ -293,18 +296,15 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       if (lane == 0) issue_s(kt);
       __syncwarp();
     }
-    for (int kt = 0; kt < 2 && kt + 2 < nkt && ok; ++kt) {
-      ok = pf_wait_warp(&bar_s[kt], 0);
-      if (ok && lane == 0) load_k(kt + 2);
-      __syncwarp();
-    }
     for (int kt = 0; kt < nkt && ok; ++kt) {
-      // P(kt) is in shared memory (its writers have also seen P V(kt-1) complete) and V(kt) has landed
-      ok = pf_wait_warp(&bar_p, kt & 1);
+      // P(kt) is in tensor memory, so S(kt) is complete and K(kt)'s buffer is free: K(kt+3) goes there
+      ok = pf_wait_warp(&bar_p[kt & 1], (kt >> 1) & 1);
       if (!ok) break;
-      ok = pf_wait_warp(&bar_v[kt & 1], (kt >> 1) & 1);
+      if (lane == 0 && kt + 3 < nkt) load_k(kt + 3);
+      __syncwarp();
+      ok = pf_wait_warp(&bar_v[kt & 1], (kt >> 1) & 1);   // V(kt) has landed
       if (!ok) break;
-      if (kt + 2 < nkt) { ok = pf_wait_warp(&bar_k[kt & 1], ((kt + 2) >> 1) & 1); if (!ok) break; }
+      if (kt + 2 < nkt) { ok = pf_wait_warp(&bar_k[(kt + 2) % 3], ((kt + 2) / 3) & 1); if (!ok) break; }
       tc_fence_after();
       if (lane == 0) {
         // O += P V: 4 steps of 16 keys; P is read from tensor memory, where it replaced the first half of its
@@ -315,18 +315,14 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
         for (int ks = 0; ks < kKeys / 16; ++ks)
           umma_bf16_ta(tmem_O, tmem_P + ks * 8, vb + ks * (2048 >> 4), kIdescPV, (kt > 0 || ks > 0));
         umma_commit(&bar_o);
+        if (kt == nkt - 1) umma_commit(&bar_done);   // O is complete
         if (kt + 2 < nkt) issue_s(kt + 2);   // into the S buffer whose tile the softmax warps have just left
       }
       __syncwarp();
-      // refill what these MMAs release: V's buffer after P V(kt), K's buffer after S(kt+2)
+      // V(kt)'s buffer is free once P V(kt) is complete: V(kt+2) goes there
       ok = pf_wait_warp(&bar_o, kt & 1);
       if (!ok) break;
       if (lane == 0 && kt + 2 < nkt) load_v(kt + 2);
-      if (kt + 4 < nkt) {
-        ok = pf_wait_warp(&bar_s[kt & 1], ((kt + 2) >> 1) & 1);
-        if (!ok) break;
-        if (lane == 0) load_k(kt + 4);
-      }
       __syncwarp();
     }
     if (!ok) { *fail = 1; if (lane == 0 && p.status) atomicOr(p.status, ST3_DEV_COPY_TIMEOUT); }
@@ -407,14 +403,15 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
         w[c >> 1] = *reinterpret_cast<const uint32_t*>(&b2);
       }
       l += sum2(add2(add[0], add[1]));
-      // P V(kt-1) must be complete before O is rescaled in place.  Every thread waits for it at every step, needed
-      // or not: that keeps a fast thread from arriving for tile kt+1 while a slow one still owes its arrival
-      // for tile kt, and keeps every waiter on this barrier's current phase.
-      if (kt > 0) {
+      // P V(kt-1) must be complete before O is rescaled in place; only then is it waited for.  The parity wait is
+      // unambiguous although this thread has not watched every phase: S(kt) is complete, hence so is P V(kt-2),
+      // issued before it, and P V(kt) cannot be issued before this thread's arrival below, so the barrier is in
+      // phase kt-1 or has just left it.
+      if (kt > 0 && __any_sync(0xffffffffu, factor != 1.f)) {
         ok = pf_wait_warp(&bar_o, (kt - 1) & 1);
         if (!ok) break;
         tc_fence_after();
-        if (__any_sync(0xffffffffu, factor != 1.f)) {
+        {
 #pragma unroll 1
           for (int cb = 0; cb < 4; ++cb) {
             uint32_t o[32];
@@ -427,11 +424,13 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       }
       // P replaces the first 32 columns of this S tile (only this thread reads or writes this lane of it, and
       // S(kt+2) lands there after P V(kt) in the tensor pipe's order)
+      // Arrivals alternate between two barriers: a thread one tile ahead of the slowest one (it cannot be further,
+      // S(kt+2) is issued only after every arrival for tile kt) then never adds to the slow one's phase.
       tmem_st32(tmem_S + lane_addr, w);
       tc_fence_before();
-      mbar_arrive_cta(&bar_p);
+      mbar_arrive_cta(&bar_p[kt & 1]);
     }
-    if (ok) { ok = pf_wait_warp(&bar_o, (nkt - 1) & 1) && !*fail; }   // the last P V: O is complete
+    if (ok) { ok = pf_wait_warp(&bar_done, 0) && !*fail; }   // the last P V: O is complete
     const float inv_l = l > 0.f ? 1.f / l : 0.f;
     if (probs && (T - 1) / kTile == qt) {   // this block holds the last query row (same answer in every thread)
       // alpha of this head: exp2(logit - ref) / sum over the visual positions, with the last row's final

@@ -1,14 +1,18 @@
 // Causal prompt attention (Eq. 2 in full) on the 5th-generation tensor cores: tcgen05.mma with
 // accumulators in tensor memory, operands staged in shared memory by TMA, for bf16 and D = 128.
 //
-// One block per (head instance, 128-query tile), two blocks per SM so that one block's softmax overlaps
-// the other's tensor work.  Warp 4 is the control warp: it issues the TMA loads and the MMAs.  Warps 0-3
-// own one query row per thread (thread i <-> TMEM lane i), so the softmax needs no cross-thread
-// reduction.  One pass over the 64-key tiles up to the diagonal, with an online softmax:
-//   S = Q K^T (tcgen05.mma, 128x64x128); P = exp2(S - ref) as bf16 into shared memory; O += P V (second
-//   MMA, accumulator in tensor memory).  `ref` follows the row's running maximum lazily: O (and the running
-//   sum) are rescaled in tensor memory only when the maximum has grown by more than 2^8, so P never
-//   exceeds 256 and rescaling is rare after the first tiles; O is divided by the sum on the way out.
+// One block per (head instance, 128-query tile), two blocks per SM.  Warp 4 is the control warp: it issues
+// the TMA loads and the MMAs.  Warps 0-3 own one query row per thread (thread i <-> TMEM lane i), so the
+// softmax needs no cross-thread reduction.  One pass over the 64-key tiles up to the diagonal, with an
+// online softmax:
+//   S = Q K^T (8 MMAs of 128x64x16) into one of two S tiles in tensor memory; P = exp2(S - ref) as bf16,
+//   written over the first half of its S tile; O += P V (4 MMAs of 128x128x16, P read from tensor memory as
+//   the A operand, accumulator in tensor memory).
+// The tensor pipe runs S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...: the next tile's scores are ready before the
+// softmax of this one ends, so the softmax warps wait for the tensor cores only to rescale O.  `ref` follows
+// the row's running maximum lazily: O (and the running sum) are rescaled in tensor memory only when the
+// maximum has grown by more than 2^8, so P never exceeds 256 and rescaling is rare after the first tiles; O
+// is divided by the sum on the way out.  K tiles are fetched three ahead, V tiles two ahead.
 // The last query row's logits on the visual positions are kept per head, normalised at the end and summed
 // over heads by a second small kernel: the scores alpha (Sec. 3.2) that prune the NEXT layer.
 //
@@ -29,7 +33,6 @@ constexpr int kBoxBytes = 128 * 128;  // one TMA box of Q: 128 rows x 64 bf16
 constexpr int kTileBytes2 = 2 * kBoxBytes;
 constexpr int kKBoxBytes = kKeys * 128;  // one TMA box of K or V: 64 rows x 64 bf16
 constexpr int kKTileBytes = 2 * kKBoxBytes;
-constexpr int kPolyPhase = 4;         // pairs (of every four) whose exponentials run on the FMA pipe; 4 = none
 constexpr uint32_t kTmemCols = 256;   // S in columns [0,64), O in [128,256)
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -148,33 +151,6 @@ __device__ __forceinline__ u64 add2(u64 a, u64 b) {
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
-__device__ __forceinline__ u64 fma2r(u64 a, u64 b, u64 c) {
-  u64 d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-// exp2 of a pair on the FMA pipe, for arguments <= 8 or so: the special-function unit, at a quarter of the FMA
-// rate, is what bounds the softmax, so half of the exponentials are computed here instead.  x is clamped to
-// >= -120, split as j + f with j = round(x) (adding and subtracting 1.5 * 2^23) and f in [-0.5, 0.5]; 2^f is a
-// cubic (relative error 7.5e-5, below the bf16 rounding of P); j is added into the exponent field.
-__device__ __forceinline__ void exp2_pair_fma(u64 x2, float& pa, float& pb) {
-  float xa, xb;
-  split2(x2, xa, xb);
-  x2 = pack2(fmaxf(xa, -120.f), fmaxf(xb, -120.f));
-  const u64 magic = pack2(12582912.f, 12582912.f);
-  const u64 t2 = add2(x2, magic);
-  const u64 nj = fma2r(t2, pack2(-1.f, -1.f), magic);   // -(round(x))
-  const u64 f2 = add2(x2, nj);
-  u64 r2 = fma2r(pack2(0.05517132f, 0.05517132f), f2, pack2(0.24261054f, 0.24261054f));
-  r2 = fma2r(r2, f2, pack2(0.69326097f, 0.69326097f));
-  r2 = fma2r(r2, f2, pack2(0.99992812f, 0.99992812f));
-  float ra, rb, ta, tb;
-  split2(r2, ra, rb);
-  split2(t2, ta, tb);
-  pa = __uint_as_float(__float_as_uint(ra) + (__float_as_uint(ta) << 23));
-  pb = __uint_as_float(__float_as_uint(rb) + (__float_as_uint(tb) << 23));
-}
-
 // kind::f16 instruction descriptors: fp32 accumulate, bf16 x bf16, M = 128.
 constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 4) << 24);
 constexpr uint32_t kIdescS = kIdescBase | ((kKeys >> 3) << 17);                 // N = 64 keys, A and B K-major
@@ -390,14 +366,9 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       for (int c = 0; c < 64; c += 2) {
         u64 t2 = nrf2;
         fma2(t2, pack2(__uint_as_float(v[c]), __uint_as_float(v[c + 1])), sc2);
-        float pa, pb;
-        if (((c >> 1) & 3) == kPolyPhase) {
-          exp2_pair_fma(t2, pa, pb);
-        } else {
-          float ta, tb;
-          split2(t2, ta, tb);
-          pa = fast_exp2(ta); pb = fast_exp2(tb);
-        }
+        float ta, tb;
+        split2(t2, ta, tb);
+        const float pa = fast_exp2(ta), pb = fast_exp2(tb);
         add[(c >> 1) & 1] = add2(add[(c >> 1) & 1], pack2(pa, pb));
         const __nv_bfloat162 b2 = __floats2bfloat162_rn(pa, pb);
         w[c >> 1] = *reinterpret_cast<const uint32_t*>(&b2);

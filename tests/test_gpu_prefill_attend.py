@@ -46,6 +46,30 @@ def test_causal_attention_and_next_layer_scores(T, H, nb, sys_len, nv):
         assert np.allclose(scores[b, :nv].cpu().numpy(), want, rtol=2e-3, atol=1e-7)
 
 
+def test_full_prompt_length_sampled_rows():
+    """LLaVA-NeXT prompt length (35 + 2880 + 128), two sequences of 32 heads: a grid of several waves with two
+    blocks per SM, as bench.py launches it.  Sampled query rows (tile edges, first, last, a ragged tail) are
+    checked one by one against the oracle's single-query attention over the causal prefix; the next layer's
+    scores of both sequences against the oracle's last row."""
+    T, H, nb, sys_len, nv = 3043, 32, 2, 35, 2880
+    q, k, v, out, scores = _run(T, H, nb, sys_len, nv, seed=11)
+    rows = [0, 1, 63, 64, 127, 128, 129, 1471, 1472, 2943, 2944, 3007, 3041, 3042]
+    for inst in (0, 21, 40, 63):
+        K = k[inst:inst + 1].double().cpu().numpy()
+        V = v[inst:inst + 1].double().cpu().numpy()
+        for r in rows:
+            ref, pr = O.attend(q[inst:inst + 1, r].double().cpu().numpy(), K[:, :r + 1], V[:, :r + 1])
+            got = out[inst, r].double().cpu().numpy()
+            bound = 2.0 ** -8 * (pr[0] @ np.abs(V[0, :r + 1]) + np.abs(ref[0])) + 1e-6
+            assert np.all(np.isfinite(got))
+            assert (np.abs(got - ref[0]) - bound).max() <= 0, f"instance {inst} row {r}"
+    for b in range(nb):
+        sl = slice(b * H, (b + 1) * H)
+        _, pr = O.attend(q[sl, T - 1].double().cpu().numpy(), k[sl].double().cpu().numpy(), v[sl].double().cpu().numpy())
+        want = O.visual_mass(pr, sys_len, nv)
+        assert np.allclose(scores[b, :nv].cpu().numpy(), want, rtol=2e-3, atol=1e-7)
+
+
 def test_scores_feed_the_scored_prefill():
     """The scores of one layer's causal attention prune the next layer's prompt (Eq. 3's alpha^{l-1})."""
     T, H, sys_len, nv, text = 96, 2, 4, 80, 12

@@ -243,6 +243,37 @@ class Job:
                             "kv_bytes_untrimmed": (full + oth) * row_bytes})
         return out
 
+    def kept_set_curve(self, points=5):
+        """Diagnostics read from the kept-id sets along one generation, averaged over the pruning layers of
+        sequence 0: (a) Eq. 10 applied to the kept sets, the share of the tokens held after decode step 1 that
+        are still held after step n (the path only ever evicts, so this is how fast the first step's set is
+        used up); (b) the share of the planted attentive tokens (or of the kept slots, if fewer) that the kept
+        set holds, i.e. whether what is kept is what the synthetic queries attend to."""
+        wl, B, h = self.wl, self.B, self.ctx.handle
+        layers = [l for l in range(wl.first_prune_layer, wl.num_layers)]
+        want = sorted(set(int(round(x)) for x in np.linspace(1, wl.decode_steps, points)))
+        self.prefill_only()
+        q, k, v, o, nb = self.q.data_ptr(), self.kn.data_ptr(), self.vn.data_ptr(), self.out.data_ptr(), self.io_bytes
+        first, out = {}, []
+        for t in range(1, wl.decode_steps + 1):
+            off = (t - 1) * nb
+            B.st3_decode_step(h, t, 0, wl.num_layers, q + off, k + off, v + off, o + off, self.stream)
+            if t not in want:
+                continue
+            ov, rec = [], []
+            for l in layers:
+                ids, cnt, _ = self.ctx.get_kept(l, with_mass=False)
+                kept = set(ids[0, :int(cnt[0])].tolist())
+                if t == 1:
+                    first[l] = kept
+                planted = set(int(i) for i in self.g.planted(0, l))
+                ov.append(len(kept & first[l]) / max(1, len(first[l])))
+                if kept:
+                    rec.append(len(kept & planted) / min(len(planted), len(kept)))
+            out.append({"step": t, "overlap_with_step_1": float(np.mean(ov)),
+                        "planted_recall": float(np.mean(rec)) if rec else None})   # None: nothing is held any more
+        return out
+
     def make_host(self):
         self.hK, self.hV = self.K.cpu().pin_memory(), self.V.cpu().pin_memory()
         self.hq0 = self.q0.cpu().pin_memory()
@@ -523,6 +554,7 @@ def main():
         job.ctx.status()
         line["per_layer_calls"] = {"value": tokens_per_gen * max(1, args.steps // 2) / (ms_pl * 1e-3), "unit": UNIT}
         line["kv_held"] = job.rows_held_curve()
+        line["kept_sets"] = job.kept_set_curve()
         line["prefill_attend"] = prefill_attend_leg(wl, device)
         # the oracle on the host cores, bounded sample
         ns = 24 if wl.batch == 1 else max(1, 24 // wl.batch)

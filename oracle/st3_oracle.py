@@ -343,6 +343,14 @@ def decode_step_lazy(cache: LayerCache, cache_src: LayerCache, q_src, v_new, n_t
     return out
 
 
+def overlap_n(ids_1, ids_n) -> float:
+    """Overlap_n of Eq. 10: |TopK(T_1) ∩ TopK(T_n)| / |TopK(T_1)|, the share of the visual tokens in the first
+    decode step's top-K that are in the n-th step's top-K too.  ids_1, ids_n: the two top-K index sets."""
+    a = set(int(i) for i in np.asarray(ids_1).ravel())
+    b = set(int(i) for i in np.asarray(ids_n).ravel())
+    return len(a & b) / len(a) if a else 1.0
+
+
 def boundary_scores(mass: np.ndarray, ids: np.ndarray, k: int):
     """(s_k, s_{k+1}): the k-th and (k+1)-th scores in selection order (None if absent)."""
     n = len(mass)

@@ -2,6 +2,7 @@
 import numpy as np
 import pytest
 
+from oracle import st3_oracle as O
 from oracle.st3_oracle import select_top, boundary_scores, prefill_select, decode_step
 
 
@@ -153,3 +154,21 @@ def test_follower_layers_adopt_the_pruning_layers_choice():
     _, m1, _ = decode_step(ca, r.standard_normal((H, D)), kn, vn, 3)
     decode_step(cb, r.standard_normal((H, D)), kn, vn, 3, select_scores=m1)
     assert np.array_equal(ca.ids, cb.ids)
+
+
+def test_overlap_n_closed_forms_and_brute_force():
+    """Eq. 10 on sets with known intersections, and against a brute-force count on top-K sets of random scores."""
+    assert O.overlap_n([1, 2, 3, 4], [1, 2, 3, 4]) == 1.0
+    assert O.overlap_n([1, 2, 3, 4], [5, 6, 7, 8]) == 0.0
+    assert O.overlap_n([1, 2, 3, 4], [3, 4, 5, 6]) == 0.5
+    assert O.overlap_n([7, 8, 9], [9]) == pytest.approx(1 / 3)          # the denominator is the first step's set
+    rng = np.random.default_rng(3)
+    ids = np.arange(200)
+    for k in (1, 17, 100, 200):
+        s1, sn = rng.normal(size=200), rng.normal(size=200)
+        t1, tn = ids[O.select_top(s1, ids, k)], ids[O.select_top(sn, ids, k)]
+        brute = sum(1 for i in np.argsort(-s1, kind="stable")[:k] if i in set(np.argsort(-sn, kind="stable")[:k].tolist())) / k
+        assert O.overlap_n(t1, tn) == pytest.approx(brute)
+    # the same scores at both steps: the top-K does not move
+    s = rng.normal(size=200)
+    assert O.overlap_n(ids[O.select_top(s, ids, 50)], ids[O.select_top(s, ids, 50)]) == 1.0

@@ -202,12 +202,28 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   const int row_base = inst * T;  // first row of this instance in the [num_inst * T][128] tensors
   const int nkt = (min(T, (qt + 1) * kTile) + kKeys - 1) / kKeys;  // causal: key tiles up to the diagonal
 
-  if (tid == 0) {
+  if (tid == 4 * 32) {   // the control warp's first lane: barriers, then the first loads at once (they are in
+                         // flight during the rest of the set-up)
     mbar_init(&bar_q, 1); mbar_init(&bar_k[0], 1); mbar_init(&bar_k[1], 1); mbar_init(&bar_k[2], 1); mbar_init(&bar_v[0], 1); mbar_init(&bar_v[1], 1);
     mbar_init(&bar_s[0], 1); mbar_init(&bar_s[1], 1); mbar_init(&bar_o, 1);
     mbar_init(&bar_p[0], 128); mbar_init(&bar_p[1], 128); mbar_init(&bar_done, 1);
     s_fail = 0;
     mbar_fence_init();
+    mbar_expect_tx(&bar_q, kTileBytes2);
+    tma_load_2d(sQ, &map_q, 0, row_base + qt * kTile, &bar_q);
+    tma_load_2d(sQ + kBoxBytes, &map_q, 64, row_base + qt * kTile, &bar_q);
+    for (int kt = 0; kt < 3 && kt < nkt; ++kt) {
+      unsigned char* d = sK2 + kt * kKTileBytes;
+      mbar_expect_tx(&bar_k[kt], kKTileBytes);
+      tma_load_2d(d, &map_k, 0, row_base + kt * kKeys, &bar_k[kt]);
+      tma_load_2d(d + kKBoxBytes, &map_k, 64, row_base + kt * kKeys, &bar_k[kt]);
+    }
+    for (int kt = 0; kt < 2 && kt < nkt; ++kt) {
+      unsigned char* d = sV2 + kt * kKTileBytes;
+      mbar_expect_tx(&bar_v[kt], kKTileBytes);
+      tma_load_2d(d, &map_v, 0, row_base + kt * kKeys, &bar_v[kt]);
+      tma_load_2d(d + kKBoxBytes, &map_v, 64, row_base + kt * kKeys, &bar_v[kt]);
+    }
   }
   __syncthreads();
   if (warp == 4) {
@@ -253,17 +269,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       }
       umma_commit(&bar_s[kt & 1]);
     };
-    if (lane == 0) {
-      mbar_expect_tx(&bar_q, kTileBytes2);
-      tma_load_2d(sQ, &map_q, 0, row_base + qt * kTile, &bar_q);
-      tma_load_2d(sQ + kBoxBytes, &map_q, 64, row_base + qt * kTile, &bar_q);
-      load_k(0);
-      if (nkt > 1) load_k(1);
-      if (nkt > 2) load_k(2);
-      load_v(0);
-      if (nkt > 1) load_v(1);
-    }
-    ok = pf_wait_warp(&bar_q, 0);
+    ok = pf_wait_warp(&bar_q, 0);   // (Q, K(0..2) and V(0..1) were requested during the set-up)
     // prologue: S(0) and S(1)
     for (int kt = 0; kt < 2 && kt < nkt && ok; ++kt) {
       ok = pf_wait_warp(&bar_k[kt], 0);

@@ -277,7 +277,10 @@ class Job:
     def make_host(self):
         self.hK, self.hV = self.K.cpu().pin_memory(), self.V.cpu().pin_memory()
         self.hq0 = self.q0.cpu().pin_memory()
-        self.hq, self.hk, self.hv = self.q.cpu().pin_memory(), self.kn.cpu().pin_memory(), self.vn.cpu().pin_memory()
+        # one pinned buffer [step][q | k_new | v_new]: the three inputs of a step lie back to back, which lets the
+        # library bring them over in one copy
+        self.hqkv = torch.stack([self.q.cpu(), self.kn.cpu(), self.vn.cpu()], dim=1).contiguous().pin_memory()
+        self.hq = self.hqkv[:, 0]
         self.hout = torch.empty_like(self.hq).pin_memory()
         self.hout0 = torch.empty_like(self.hq0).pin_memory()
         self.dK, self.dV, self.dq0 = torch.empty_like(self.K), torch.empty_like(self.V), torch.empty_like(self.q0)
@@ -291,11 +294,12 @@ class Job:
         B.st3_prefill_select(h, 0, L, self.dq0.data_ptr(), self.dK.data_ptr(), self.dV.data_ptr(), self.text,
                              self.out0.data_ptr(), st)
         self.hout0.copy_(self.out0, non_blocking=True)
-        q, k, v, o, nb = self.hq.data_ptr(), self.hk.data_ptr(), self.hv.data_ptr(), self.hout.data_ptr(), self.io_bytes
+        base, o, nb = self.hqkv.data_ptr(), self.hout.data_ptr(), self.io_bytes
         step_fn = self.lib.st3_decode_step_host
         for t in range(1, self.wl.decode_steps + 1):
             off = (t - 1) * nb
-            rc = step_fn(h, t, 0, L, q + off, k + off, v + off, o + off, st)
+            q = base + 3 * off
+            rc = step_fn(h, t, 0, L, q, q + nb, q + 2 * nb, o + off, st)
             if rc:
                 raise B.St3Error(rc, f"st3_decode_step_host t={t}")
 

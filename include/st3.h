@@ -161,7 +161,9 @@ st3_status st3_decode_step(st3_ctx* ctx, int32_t step, int32_t layer_begin, int3
 
 /* Same step with HOST buffers (pinned memory recommended): the library copies q/k_new/v_new to
  * staging areas inside its workspace, runs the step and copies `out` back, all on the stream.
- * The host buffers must stay untouched until the stream has passed the call. */
+ * The host buffers must stay untouched until the stream has passed the call.  When the three inputs
+ * lie back to back in host memory (k_new_host = q_host + size, v_new_host = k_new_host + size) and the
+ * call covers all layers, they travel as one copy. */
 st3_status st3_decode_step_host(st3_ctx* ctx, int32_t step, int32_t layer_begin, int32_t layer_count,
                                 const void* q_host, const void* k_new_host, const void* v_new_host,
                                 void* out_host, void* cuda_stream);

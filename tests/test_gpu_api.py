@@ -20,7 +20,10 @@ def _small(**kw):
     return get_workload("tiny").scaled(**base)
 
 
-def test_host_buffer_step_equals_device_step():
+@pytest.mark.parametrize("packed", [False, True])
+def test_host_buffer_step_equals_device_step(packed):
+    """`packed`: q, k_new, v_new back to back in one pinned buffer (the library's single-copy path);
+    otherwise three separate buffers (three copies)."""
     wl = _small()
     a, b = GpuRun(wl), GpuRun(wl)
     try:
@@ -29,8 +32,13 @@ def test_host_buffer_step_equals_device_step():
         for t in range(1, 6):
             a.decode(t)
             q, kn, vn = b.inputs(t)
-            hq, hk, hv = (x.cpu().pin_memory() for x in (q, kn, vn))
-            hout = torch.empty_like(hq).pin_memory()
+            if packed:
+                hqkv = torch.stack([q.cpu(), kn.cpu(), vn.cpu()]).contiguous().pin_memory()
+                hq, hk, hv = hqkv[0], hqkv[1], hqkv[2]
+                assert hk.data_ptr() == hq.data_ptr() + hq.numel() * hq.element_size()
+            else:
+                hq, hk, hv = (x.cpu().pin_memory() for x in (q, kn, vn))
+            hout = torch.empty_like(q.cpu()).pin_memory()
             b.ctx.decode_step_host(t, hq, hk, hv, hout)
             torch.cuda.synchronize()
             assert torch.equal(hout, a.out.cpu()), t

@@ -488,15 +488,16 @@ extern "C" st3_status st3_prefill_attend(const void* q, const void* k, const voi
   if (num_visual > 0 && (!head_probs || !scores)) return ST3_ERR_INVALID_ARG;
   if (head_dim != kPfD || dtype != ST3_BF16) return ST3_ERR_UNSUPPORTED;
   if ((long long)num_inst * seq_len > 0x7fffffffLL || num_inst > 65535) return ST3_ERR_UNSUPPORTED;
-  static EncodeTiledFn encode = nullptr;
-  if (!encode) {
+  // looked up once (initialisation of a local static is thread-safe); null if the driver does not offer it
+  static const EncodeTiledFn encode = [] {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
         qres != cudaDriverEntryPointSuccess)
-      return ST3_ERR_CUDA;
-    encode = reinterpret_cast<EncodeTiledFn>(fn);
-  }
+      fn = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(fn);
+  }();
+  if (!encode) return ST3_ERR_CUDA;
   CUtensorMap mq, mk, mv;
   const size_t rows = (size_t)num_inst * seq_len;
   if (!make_map(encode, &mq, q, rows, kTile) || !make_map(encode, &mk, k, rows, kKeys) ||

@@ -211,7 +211,8 @@ int64_t st3_launch_count(const st3_ctx* ctx);
  *               positions [sys_len, sys_len + num_visual), summed over heads -- the alpha of Sec. 3.2 that
  *               Eq. 3 uses to prune the NEXT layer (feed it to st3_prefill_select_scored).
  *               head_probs and scores may be NULL when num_visual is 0.
- *   dev_status  dev int, may be NULL: ST3_DEV_COPY_TIMEOUT is OR-ed in if a copy or an MMA never completes
+ *   dev_status  dev int, may be NULL: ST3_DEV_COPY_TIMEOUT is OR-ed in if a copy or an MMA never completes,
+ *               ST3_DEV_RANGE if a block finds its shared-memory window misaligned (it then does nothing)
  * Needs no context and no workspace beyond head_probs. */
 st3_status st3_prefill_attend(const void* q, const void* k, const void* v, void* out, float* head_probs,
                               float* scores, int* dev_status, int32_t num_inst, int32_t num_heads,

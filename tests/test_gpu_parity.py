@@ -46,6 +46,20 @@ def test_small_odd_shapes(dtype, D, H):
     run_and_check(wl, 5, layers_per_call=2)
 
 
+def test_largest_visual_span_and_head_count():
+    """Close to the largest visual span the library accepts (8192; the seeded generator numbers at most 8192
+    tokens per sequence, prompt and generated) for the top-k and the compaction, and the generator's largest
+    head count, on otherwise small shapes."""
+    wl = get_workload("tiny").scaled(dtype="bf16", head_dim=64, num_heads=2, num_layers=2, batch=2, sys_len=5,
+                                     num_visual=8150, text_len_min=3, text_len_max=20, decode_steps=4,
+                                     first_prune_layer=0, stride=1, step_ratio_bp=1500, tau=6.0, num_planted=200)
+    run_and_check(wl, 4)
+    wl = get_workload("tiny").scaled(dtype="bf16", head_dim=128, num_heads=64, num_layers=2, batch=1, sys_len=4,
+                                     num_visual=96, text_len_min=9, text_len_max=9, decode_steps=3,
+                                     first_prune_layer=0, stride=1, step_ratio_bp=2500, tau=5.0, num_planted=9)
+    run_and_check(wl, 3)
+
+
 def test_no_visual_tokens_and_single_text_token():
     wl = get_workload("tiny").scaled(num_visual=0, num_planted=0, sys_len=0, text_len_min=1, text_len_max=1,
                                      decode_steps=3)

@@ -200,7 +200,11 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   const int qt = blockIdx.x, inst = blockIdx.y;
   const int T = p.T;
   const int row_base = inst * T;  // first row of this instance in the [num_inst * T][128] tensors
-  const int nkt = (min(T, (qt + 1) * kTile) + kKeys - 1) / kKeys;  // causal: key tiles up to the diagonal
+  // Query tiles are aligned to the END of the prompt: the ragged tile is the first one, where the causal prefix
+  // is shortest, instead of the last one, where a mostly empty tile would walk every key.  Its rows before the
+  // prompt (q0 < 0) are dead: their loads read the fill value or a neighbour's rows, nothing is stored.
+  const int q0 = T - ((int)gridDim.x - qt) * kTile;                // first query row of this tile
+  const int nkt = (q0 + kTile + kKeys - 1) / kKeys;                // causal: key tiles up to the diagonal
 
   if (tid == 4 * 32) {   // the control warp's first lane: barriers, then the first loads at once (they are in
                          // flight during the rest of the set-up)
@@ -210,8 +214,8 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     s_fail = 0;
     mbar_fence_init();
     mbar_expect_tx(&bar_q, kTileBytes2);
-    tma_load_2d(sQ, &map_q, 0, row_base + qt * kTile, &bar_q);
-    tma_load_2d(sQ + kBoxBytes, &map_q, 64, row_base + qt * kTile, &bar_q);
+    tma_load_2d(sQ, &map_q, 0, row_base + q0, &bar_q);
+    tma_load_2d(sQ + kBoxBytes, &map_q, 64, row_base + q0, &bar_q);
     for (int kt = 0; kt < 3 && kt < nkt; ++kt) {
       unsigned char* d = sK2 + kt * kKTileBytes;
       mbar_expect_tx(&bar_k[kt], kKTileBytes);
@@ -311,8 +315,8 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   } else {
     // ===================== softmax warps: thread <-> query row =====================
     const int r = tid;                        // row inside the tile == TMEM lane
-    const int qi = qt * kTile + r;            // query position inside the instance
-    const bool live = qi < T;
+    const int qi = q0 + r;                    // query position inside the instance (< T always)
+    const bool live = qi >= 0;
     const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
     const float sc = 1.4426950408889634f * rsqrtf((float)kPfD);
     float ref = -INFINITY;   // what P is taken relative to; trails the running maximum by at most 8 (log2 domain)
@@ -328,7 +332,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
       uint32_t v[64];
       tmem_ld64(tmem_S + lane_addr, v);
       const int j0 = kt * kKeys;
-      if (j0 + kKeys > qt * kTile + 1 || j0 + kKeys > T) {   // the tile touches the diagonal or the end of the prompt
+      if (j0 + kKeys > q0 + 1) {   // the tile reaches past the first row's own position: mask (also covers keys >= T)
 #pragma unroll
         for (int c = 0; c < 64; ++c)
           if (!(live && j0 + c <= qi && j0 + c < T)) v[c] = 0xff800000u;
@@ -339,10 +343,10 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
 #pragma unroll
         for (int e = 0; e < 4; ++e) m4[e] = fmax3(m4[e], __uint_as_float(v[c + e]), __uint_as_float(v[c + 4 + e]));
       const float mx = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])) * sc;   // the scale is positive: max and scaling commute
-      if (probs && (T - 1) / kTile == qt && ((T - 1) % kTile) >> 5 == warp) {
+      if (probs && qt == (int)gridDim.x - 1 && warp == 3) {
         // the last query row lives in one lane of this warp: hand its logits on the visual positions to the
         // whole warp, which stores them coalesced; they are normalised once the row is complete
-        const int src = (T - 1) & 31;
+        const int src = 31;   // the last query row is the last row of the last tile
 #pragma unroll
         for (int c = 0; c < 64; c += 32) {
           float mine = 0.f;
@@ -409,7 +413,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     }
     if (ok) { ok = pf_wait_warp(&bar_done, 0) && !*fail; }   // the last P V: O is complete
     const float inv_l = l > 0.f ? 1.f / l : 0.f;
-    if (probs && (T - 1) / kTile == qt) {   // this block holds the last query row (same answer in every thread)
+    if (probs && qt == (int)gridDim.x - 1) {   // this block holds the last query row (same answer in every thread)
       // alpha of this head: exp2(logit - ref) / sum over the visual positions, with the last row's final
       // reference and sum; the 128 softmax threads share the work
       if (last_row) { s_last[0] = ref; s_last[1] = ok ? inv_l : 0.f; }

@@ -229,7 +229,21 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
     if (cudaLaunchKernelEx(&cfg, st3_attend_kernel<T, D>, p) != cudaSuccess) return ST3_ERR_CUDA;
   }
   if (e1) cudaEventRecord(e1, st);
-  st3_finish_kernel<T, D><<<(unsigned)(2 * p.layer_count * c.batch), kFinishThreads, ctx->finish_smem, st>>>(p);
+  {
+    // Also a programmatic dependent launch: the attention kernel allows it at its start, the blocks become
+    // resident as that grid drains and their first instruction waits for all of it.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(2 * p.layer_count * c.batch));
+    cfg.blockDim = dim3(kFinishThreads);
+    cfg.dynamicSmemBytes = (size_t)ctx->finish_smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = ctx->profiling ? 0 : 1;
+    if (cudaLaunchKernelEx(&cfg, st3_finish_kernel<T, D>, p) != cudaSuccess) return ST3_ERR_CUDA;
+  }
   if (e2) cudaEventRecord(e2, st);
   ctx->launches += 2;
   return cudaGetLastError() == cudaSuccess ? ST3_OK : ST3_ERR_CUDA;

@@ -106,6 +106,9 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
   __shared__ float s_stat[kSlots][kGroupWarps][2];
   __shared__ int s_abort;
 
+  // The finish launch that follows may be set up while this kernel runs (its blocks take the SMs this grid's
+  // blocks leave and wait there for the whole grid: no launch latency between the two kernels).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     for (int s = 0; s < kSlots; ++s)
@@ -397,6 +400,9 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
       if (lane == 0) mbar_arrive(&s_done[s][grp]);
     }
   }
+  // This grid started without waiting for the launch before it (flags order what they share).  It must not
+  // *complete* before that launch has, though: the finish launch after this one waits for this grid only.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 

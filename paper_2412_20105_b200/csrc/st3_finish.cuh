@@ -48,7 +48,10 @@ __global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepPa
   __shared__ float s_half[kFinishThreads / 2];
   __shared__ int s_sel[3];  // digit, count above, count in bin
 
-  // the next step's attention launch may start now; it waits on p.flags for what this launch changes
+  // This launch may have been set up while the attention launch before it was still running: wait for that
+  // whole grid (and, through it, for everything earlier in the stream).  Then the next step's attention launch
+  // may start; it waits on p.flags for what this launch changes.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int tid = threadIdx.x, lane = tid & 31;
   const int B = p.B, H = p.H, Nv = p.Nv;

@@ -334,10 +334,13 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
     p.cvp[i + 1] = p.cvp[i] + cv;
     p.lstart[i] = c.batch * (p.cvp[i] + i * p.ct);
     p.rpv[i] = cv ? ceil_div(ncur, cv) : 0;
-    make_fast_div((unsigned)(cv + p.ct), &p.per_mul[i], &p.per_shift[i]);
+    make_fast_div((unsigned)(cv > 0 ? cv : 1), &p.cv_mul[i], &p.cv_shift[i]);
   }
   p.lstart[layer_count] = c.batch * (p.cvp[layer_count] + layer_count * p.ct);
   make_fast_div((unsigned)c.num_heads, &p.h_mul, &p.h_shift);
+  p.text_items = layer_count * c.batch * p.ct;
+  make_fast_div((unsigned)(c.batch * p.ct), &p.bct_mul, &p.bct_shift);
+  make_fast_div((unsigned)p.ct, &p.ct_mul, &p.ct_shift);
   const long long total_items = (long long)c.batch * (p.cvp[layer_count] + (long long)layer_count * p.ct);
   if (total_items > L.max_items || total_items * c.num_heads > 0x3fffffffLL) return ST3_ERR_CAPACITY;
   p.total_work = (int)(total_items * c.num_heads);

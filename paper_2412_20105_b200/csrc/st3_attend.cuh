@@ -142,7 +142,7 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
       T *newK, *newV;
       uint4 nv[NV];
     };
-    int lcur = 0;  // layer of the previous item: this warp's items arrive in increasing order
+    int lcur = 0;  // layer of the previous visual item: this warp's items arrive in increasing order
     long long lb_ready = -1;  // the (l, b) whose visual rows were last seen released by the previous finish launch
     // the first item of every manager is fixed (no round trip to the counter before the first copy);
     // the counter starts behind those and hands out the rest
@@ -154,16 +154,33 @@ __global__ void __launch_bounds__(kAttendThreads, 2) st3_attend_kernel(const Ste
       if (!d.valid) return;
       if (lane == 0)  // prefetch the index after this one
         x_next = p.first_dynamic + (int)(atomicAdd(reinterpret_cast<unsigned*>(p.work_counter), 1u) - p.counter_base);
-      const int item = (int)fast_div((unsigned)x, p.h_mul, p.h_shift);
-      const int h = x - item * H;
-      while (lcur + 1 < p.layer_count && item >= p.lstart[lcur + 1]) ++lcur;
-      const int l_rel = lcur, l = p.layer_begin + l_rel;
-      const int cv = p.cvp[l_rel + 1] - p.cvp[l_rel];
-      const int per = cv + p.ct;
-      const int off = item - p.lstart[l_rel];
-      const int b = (int)fast_div((unsigned)off, p.per_mul[l_rel], p.per_shift[l_rel]);
-      const int c = off - b * per;
-      const bool is_vis = c < cv;
+      // Order of work: the text (and system) chunks of every layer first, then the visual chunks layer by
+      // layer.  Only visual rows are moved by the previous step's finish launch, which is still running when
+      // this launch starts: what does not depend on it comes first (+4 % tokens/s at B=1 over a layer-major
+      // order, whose visual chunks of the first pruning layers waited ~4 us each for their flag).  A partial's
+      // slot keeps the layer-major numbering (visual chunks, then text chunks of each (l, b)) that the finish
+      // kernel reads.
+      const int xi = (int)fast_div((unsigned)x, p.h_mul, p.h_shift);
+      const int h = x - xi * H;
+      const bool is_vis = xi >= p.text_items;
+      int l_rel, b, c, cv;
+      if (!is_vis) {
+        l_rel = (int)fast_div((unsigned)xi, p.bct_mul, p.bct_shift);
+        const int rem = xi - l_rel * p.B * p.ct;
+        b = (int)fast_div((unsigned)rem, p.ct_mul, p.ct_shift);
+        cv = p.cvp[l_rel + 1] - p.cvp[l_rel];
+        c = cv + rem - b * p.ct;
+      } else {
+        const int iv = xi - p.text_items;
+        while (lcur + 1 < p.layer_count && iv >= p.B * p.cvp[lcur + 1]) ++lcur;
+        l_rel = lcur;
+        cv = p.cvp[l_rel + 1] - p.cvp[l_rel];
+        const int off = iv - p.B * p.cvp[l_rel];
+        b = (int)fast_div((unsigned)off, p.cv_mul[l_rel], p.cv_shift[l_rel]);
+        c = off - b * cv;
+      }
+      const int l = p.layer_begin + l_rel;
+      const int item = p.lstart[l_rel] + b * (cv + p.ct) + c;
       int seg_rows, rows_per, ci;
       if (is_vis) {
         seg_rows = p.ncur[l_rel]; rows_per = p.rpv[l_rel]; ci = c;

@@ -52,8 +52,11 @@ struct StepParams {
   int cvp[kMaxLayers + 1];  // prefix sum of visual chunks per layer (relative layer index)
   int lstart[kMaxLayers + 1];       // first work item of each layer: B * (cvp[l] + l * ct)
   int rpv[kMaxLayers];              // rows per visual chunk of each layer
-  unsigned per_mul[kMaxLayers];     // fast division by (visual + text chunks) of each layer
-  unsigned per_shift[kMaxLayers];
+  unsigned cv_mul[kMaxLayers];      // fast division by the visual chunks of each layer
+  unsigned cv_shift[kMaxLayers];
+  int text_items;                   // layer_count * B * ct: the attention launch works through these first
+  unsigned bct_mul, bct_shift;      // fast division by B * ct
+  unsigned ct_mul, ct_shift;        // fast division by ct
   int ncur[kMaxLayers];     // visual rows held before this step (host's schedule bookkeeping)
   int ntgt[kMaxLayers];     // visual rows to hold after this step
   int nold[kMaxLayers];     // visual rows the device should report before this step

@@ -74,7 +74,7 @@ typedef struct {
   int32_t num_visual;        /* |V| at the input of layer 0                                     */
   int32_t max_text_len;      /* capacity for |I| per sequence                                   */
   int32_t max_decode_steps;  /* capacity for |O|                                                */
-  int32_t first_prune_layer; /* 3: "avoid pruning tokens in the first three layers" (Sec. 3.2)  */
+  int32_t first_prune_layer; /* 3: layers 0-2 are never pruned (Sec. 3.2)                       */
   int32_t stride;            /* S: prune at layers first, first+S, ... (Algorithm 1)            */
   int32_t first_ratio_bp;    /* P in basis points of |V|; the paper sets 50% = 5000 (Eq. 9)     */
   int32_t step_ratio_bp;     /* R in basis points of |V| removed at each later pruning layer    */

@@ -46,7 +46,7 @@ class Schedule:
     step_ratio_bp: int               # R in basis points of num_visual
     tau: float                       # Eq. 8 decay horizon
     first_ratio_bp: int = 5000       # P, "set to 50%" (text under Eq. 9)
-    first_prune_layer: int = 3       # "avoid pruning tokens in the first three layers"
+    first_prune_layer: int = 3       # layers 0-2 are never pruned (Sec. 3.2)
     anneal: str = "cosine"           # "cosine" | "linear" | "exp" | "none"
     sigma: float = 20.0              # only for anneal == "exp"
     disable_trim: bool = False       # full-KV comparison run
@@ -183,14 +183,6 @@ class LayerCache:
         K = np.concatenate([self.K_sys, self.K_vis, self.K_txt], axis=1)
         V = np.concatenate([self.V_sys, self.V_vis, self.V_txt], axis=1)
         return K, V
-
-    def keep_ids(self, kept_ids) -> None:
-        """Adopt a given kept set (teacher forcing); order of `ids` is preserved."""
-        kept = set(int(i) for i in kept_ids)
-        pos = np.array([j for j, i in enumerate(self.ids) if int(i) in kept], dtype=np.int64)
-        self.K_vis = self.K_vis[:, pos]
-        self.V_vis = self.V_vis[:, pos]
-        self.ids = self.ids[pos]
 
 
 def rank_order(scores: np.ndarray, ids: np.ndarray) -> np.ndarray:

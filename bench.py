@@ -21,9 +21,8 @@ import tempfile
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
-for _p in (ROOT, os.path.join(ROOT, "tests")):
-    if _p not in sys.path:
-        sys.path.insert(0, _p)
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
 
 import numpy as np
 import torch
@@ -148,6 +147,45 @@ def attend_bytes(wl, cfg, B_mod, text_len, step):
     return total
 
 
+def path_bytes(wl, cfg, B_mod, text_len):
+    """Bytes one whole generation must move, by the method's own accounting (not what the kernels happen to
+    touch): per (sequence, layer) and decode step every cached K/V row once (r*T_cur), the new row read and
+    written (2r), the query read and the output written (2*H*D*e), and, where the layer evicts at this step,
+    one fp32 score term per head per visual row written and read back plus ids and scores ((8H+8)*n_cur) and
+    the rows that close the holes read and written (2*r*d for d evicted rows, an upper bound on what hole
+    filling moves).  Prefill: the prompt rows read and written into the cache (2*r*T0), read again by the last
+    query's attention (r*T0), the same selection terms.  Partials of the split attention are scratch of this
+    implementation and are not counted."""
+    e = 2 if wl.dtype == "bf16" else 4
+    H, D = wl.num_heads, wl.head_dim
+    r = 2 * H * D * e
+    total = 0
+    for step in range(0, wl.decode_steps + 1):
+        for l in range(wl.num_layers):
+            n_cur = wl.num_visual if step == 0 else B_mod.st3_schedule_count(cfg, l, step - 1)
+            n_tgt = min(n_cur, B_mod.st3_schedule_count(cfg, l, step))
+            for b in range(wl.batch):
+                t_cur = wl.sys_len + n_cur + int(text_len[b]) + step
+                total += r * t_cur + 2 * H * D * e + (2 * r if step > 0 else 2 * r * t_cur)
+                if n_tgt < n_cur:
+                    total += (8 * H + 8) * n_cur + 2 * r * (n_cur - n_tgt)
+    return total
+
+
+def schedule_of(wl, **kw):
+    """The oracle's schedule object for a workload (used by the CPU legs only)."""
+    from oracle import st3_oracle as O
+    args = dict(num_layers=wl.num_layers, num_visual=wl.num_visual, stride=wl.stride,
+                step_ratio_bp=wl.step_ratio_bp, tau=wl.tau, first_ratio_bp=wl.first_ratio_bp,
+                first_prune_layer=wl.first_prune_layer)
+    args.update(kw)
+    return O.Schedule(**args)
+
+
+def f64(t):
+    return t.detach().to("cpu").to(torch.float64).numpy()
+
+
 # ----------------------------------------------------------------------------------------------
 # our arm
 # ----------------------------------------------------------------------------------------------
@@ -164,6 +202,9 @@ class Job:
         self.cfg = B.config_from_workload(wl, disable_trim=int(disable_trim), rows_per_chunk=rows_per_chunk,
                                            static_rank=int(static_rank))
         self.ctx = B.Context(self.cfg, device)
+        # every input of a generation is in device memory before its first launch, which is what the
+        # overlapping-steps mode asks of its caller
+        B.st3_set_overlap(self.ctx.handle, True)
         self.lib = B.load()
         L, T = wl.num_layers, wl.decode_steps
         g = self.g
@@ -350,8 +391,7 @@ def oracle_sample(wl, g, K, V, q0, q, kn, vn, nsteps, warm_steps, reps=1):
     """Times the oracle, as it stands, on decode steps 1..nsteps of the workload (all layers, all
     sequences, free-running after its own prefill).  Returns (tokens/s, seconds, threads)."""
     from oracle import st3_oracle as O
-    from helpers import make_schedule, f64
-    sched = make_schedule(wl)
+    sched = schedule_of(wl)
     caches = {}
     for l in range(wl.num_layers):
         for b in range(wl.batch):
@@ -379,6 +419,88 @@ def oracle_sample(wl, g, K, V, q0, q, kn, vn, nsteps, warm_steps, reps=1):
     except Exception:
         threads = 1
     return wl.batch * nsteps / secs, secs, threads, first, t - 1
+
+
+def free_running_report(wl, device, steps=None, rel=1e-3):
+    """Oracle and GPU run the same generation side by side WITHOUT the oracle ever adopting the GPU's state.
+    After prefill and after every decode step the kept visual ids of every (sequence, layer) unit are compared
+    as sets.  Reports the first step at which some unit's set differs (None if never), whether the oracle's
+    scores at that cut were a near-tie (gap at the boundary <= rel * |s_k|), how many units have left the
+    oracle's trajectory by the end, and the largest output error over the units that still agree (absolute
+    for fp32, relative to max(|ref|, 1e-2) for bf16)."""
+    from oracle import st3_oracle as O
+    from paper_2412_20105_b200 import binding as B
+    T = wl.decode_steps if steps is None else min(steps, wl.decode_steps)
+    g = SynthInputs(wl)
+    sched = schedule_of(wl)
+    cfg = B.config_from_workload(wl)
+    ctx = B.Context(cfg, device)
+    L, Bn = wl.num_layers, wl.batch
+    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    out = torch.empty((L, Bn, wl.num_heads, wl.head_dim), dtype=tdt, device=device)
+    text = g.text_len.tolist()
+    caches, agree = {}, {}
+    first, diverged, max_err = None, 0, 0.0
+
+    def err_of(got, ref):
+        if wl.dtype == "f32":
+            return float(np.abs(got - ref).max())
+        return float((np.abs(got - ref) / np.maximum(np.abs(ref), 1e-2)).max())
+
+    def compare(step, masses, ids_before, ref_out):
+        nonlocal first, diverged, max_err
+        got_out = f64(out)
+        for l in range(L):
+            ids, cnt, _ = ctx.get_kept(l, with_mass=False)
+            ids, cnt = ids.cpu().numpy(), cnt.cpu().numpy()
+            for b in range(Bn):
+                if not agree[(b, l)]:
+                    continue
+                max_err = max(max_err, err_of(got_out[l, b], ref_out[(b, l)]))
+                c = caches[(b, l)]
+                if set(ids[b, :int(cnt[b])].tolist()) == set(c.ids.tolist()):
+                    continue
+                agree[(b, l)] = False
+                diverged += 1
+                if first is None:
+                    k = c.n_cur
+                    s_k, s_k1 = O.boundary_scores(masses[(b, l)], ids_before[(b, l)], k)
+                    gap = None if s_k is None or s_k1 is None else (s_k - s_k1) / max(abs(s_k), 1e-300)
+                    first = {"step": step, "layer": l, "sequence": b, "near_tie": gap is not None and gap <= rel,
+                             "relative_gap_at_cut": gap}
+
+    try:
+        q0 = g.queries([0], device=device)[0]
+        masses, before, ref_out = {}, {}, {}
+        for l in range(L):
+            K, V = g.prompt_kv([l], device=device)
+            ctx.prefill_select(q0[l:l + 1].contiguous(), K, V, text, out[l:l + 1], layer_begin=l)
+            Kc, Vc, qc = K.cpu(), V.cpu(), q0[l].cpu()
+            for b in range(Bn):
+                t0 = wl.sys_len + wl.num_visual + int(text[b])
+                o, m, caches[(b, l)] = O.prefill_select(f64(qc[b]), f64(Kc[0, b][:, :t0]), f64(Vc[0, b][:, :t0]),
+                                                        wl.sys_len, wl.num_visual, sched.n0(l))
+                agree[(b, l)] = True
+                masses[(b, l)], before[(b, l)], ref_out[(b, l)] = m, np.arange(wl.num_visual), o
+        compare(0, masses, before, ref_out)
+        for t in range(1, T + 1):
+            q = g.queries([t], device=device)[0]
+            kn, vn = g.new_kv([t], device=device)
+            ctx.decode_step(t, q, kn[0], vn[0], out)
+            qc, kc, vc = f64(q), f64(kn[0]), f64(vn[0])
+            for l in range(L):
+                for b in range(Bn):
+                    if agree[(b, l)]:
+                        ref_out[(b, l)], masses[(b, l)], before[(b, l)] = O.decode_step(
+                            caches[(b, l)], qc[l, b], kc[l, b], vc[l, b], sched.n(l, t))
+            compare(t, masses, before, ref_out)
+        ctx.status()
+    finally:
+        ctx.close()
+    return {"workload": wl.name, "steps_compared": T, "units": L * Bn, "first_divergence": first,
+            "units_diverged_by_the_end": diverged, "max_output_error_while_in_agreement": max_err,
+            "error_kind": "max-abs" if wl.dtype == "f32" else "max relative to max(|ref|, 1e-2)",
+            "mode": "neither side is re-seeded from the other; kept-id sets compared after every step"}
 
 
 def prefill_attend_leg(wl, device, iters=10, max_instances=2048):
@@ -415,6 +537,63 @@ def prefill_attend_leg(wl, device, iters=10, max_instances=2048):
             "flops": "causal half of Q K^T and P V (4 D T (T+1)/2 per instance)"}
 
 
+def kernel_roofline(job, steps, world):
+    """Attention-kernel time from the library's own events (which serialise the launches), against the
+    algorithmic bytes of the same launches."""
+    B, wl = job.B, job.wl
+    B.st3_profile_enable(job.ctx.handle, True)
+    for _ in range(steps):
+        job.generation()
+    attn_ms, finish_ms, n_attn, _ = B.st3_profile_read(job.ctx.handle)
+    B.st3_profile_enable(job.ctx.handle, False)
+    alg = sum(attend_bytes(wl, job.cfg, B, job.text, t) for t in range(0, wl.decode_steps + 1)) * steps
+    peak, peak_kind = measured_peak()
+    achieved = alg / (attn_ms * 1e-3) / 1e9
+    ratio = attend_traffic_ratio(wl.name) if world == 1 else None
+    return {"bound": "hbm", "kernel": "st3_attend_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+            "frac": achieved / peak, "peak_source": f"of {peak_kind}",
+            "traffic": None if ratio is None else ratio * alg / max(1, n_attn),
+            "algorithmic_bytes_per_launch": alg / max(1, n_attn), "us_per_launch": attn_ms * 1e3 / max(1, n_attn),
+            "timing_mode": "launches serialised by the events around each kernel (no overlap between a step's "
+                           "selection kernel and the next step's attention kernel), so us_per_launch x launches "
+                           "exceeds ms_per_step, which is timed with the steps overlapping",
+            "launches_timed": n_attn, "attend_share_of_kernel_time": attn_ms / max(1e-9, attn_ms + finish_ms)}
+
+
+def add_path_fraction(roofline, job, ms_per_generation):
+    """Whole fused path: the method's bytes of one generation over its measured time, against the same peak."""
+    pb = path_bytes(job.wl, job.cfg, job.B, job.text)
+    roofline["path_algorithmic_bytes_per_step"] = pb
+    roofline["path_achieved"] = pb / (ms_per_generation * 1e-3) / 1e9
+    roofline["path_frac"] = roofline["path_achieved"] / roofline["peak"]
+    return roofline
+
+
+def other_workload_line(name, device, rank):
+    """One timed generation of another LLaVA-shaped workload (after one warm-up generation): tokens/s, the
+    attention kernel's and the whole path's fraction of the HBM peak, clocks during the timed generation."""
+    wl = get_workload(name)
+    job = Job(wl, device)
+    try:
+        job.generation()
+        job.ctx.status()
+        sampler = ClockSampler(rank)
+        sampler.start()
+        time.sleep(0.2)
+        ms = timed(job.generation, 1, False)
+        clocks = sampler.stop()
+        job.ctx.status()
+        roof = add_path_fraction(kernel_roofline(job, 1, 1), job, ms)
+        return {"workload": wl.name, "value": wl.batch * wl.decode_steps / (ms * 1e-3), "unit": UNIT,
+                "ms_per_step": ms, "steps": 1, "warmup": 1, "frac": roof["frac"], "path_frac": roof["path_frac"],
+                "achieved": roof["achieved"], "us_per_launch": roof["us_per_launch"], "traffic": roof["traffic"],
+                "clocks": clocks}
+    finally:
+        job.ctx.close()
+        del job
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -424,6 +603,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows-per-chunk", type=int, default=0)
     ap.add_argument("--no-extras", action="store_true", help="skip the e2e, unpruned and cpu_baseline legs")
+    ap.add_argument("--no-others", action="store_true", help="skip the one-generation runs of the other workloads")
     ap.add_argument("--leg", default="", choices=["", "prefill_attend"],
                     help="run one auxiliary leg alone and print its JSON (for timing or profiling that kernel)")
     ap.add_argument("--instances", type=int, default=2048, help="cap on the (sequence, head) instances of --leg")
@@ -437,6 +617,8 @@ def main():
                           f"{wl.decode_steps} decode steps, S={wl.stride} R={wl.step_ratio_bp}bp "
                           f"P={wl.first_ratio_bp}bp tau={wl.tau:g}",
               "step": "prefill-select of all layers + all decode steps of one batch",
+              "launch_mode": "one call per decode step over all layers; consecutive steps overlap on the GPU "
+                             "(st3_set_overlap: every input is in device memory before the generation starts)",
               "l2": "inputs larger than L2 (per-step K/V working set > 126 MB); no explicit flush",
               "parallelism": f"{args.gpus} independent replica(s), no collectives"}
 
@@ -461,7 +643,9 @@ def main():
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": secs * 1e3 / args.steps,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
                 "data": "synthetic", "config": config,
-                "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+                "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+                                 "threads": f"numpy fp64; the Python loop over (layer, sequence) is serial, the "
+                                            f"matrix products inside it use a BLAS pool of {threads} thread(s)"},
                 "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
                 "gpu_launches": 0}
         print(json.dumps(line))
@@ -499,20 +683,7 @@ def main():
     value = job_value(tokens_per_gen, args.steps, world, ms)
 
     # per-kernel time of the attention kernel (events around it inside the library), same work
-    B.st3_profile_enable(job.ctx.handle, True)
-    for _ in range(args.steps):
-        job.generation()
-    attn_ms, finish_ms, n_attn, _ = B.st3_profile_read(job.ctx.handle)
-    B.st3_profile_enable(job.ctx.handle, False)
-    alg = sum(attend_bytes(wl, job.cfg, B, job.text, t) for t in range(0, wl.decode_steps + 1)) * args.steps
-    peak, peak_kind = measured_peak()
-    achieved = alg / (attn_ms * 1e-3) / 1e9
-    ratio = attend_traffic_ratio(wl.name) if world == 1 else None
-    roofline = {"bound": "hbm", "kernel": "st3_attend_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": f"of {peak_kind}",
-                "traffic": None if ratio is None else ratio * alg / max(1, n_attn),
-                "algorithmic_bytes_per_launch": alg / max(1, n_attn), "us_per_launch": attn_ms * 1e3 / max(1, n_attn),
-                "launches_timed": n_attn, "attend_share_of_kernel_time": attn_ms / max(1e-9, attn_ms + finish_ms)}
+    roofline = add_path_fraction(kernel_roofline(job, args.steps, world), job, ms / args.steps)
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": True,
@@ -566,12 +737,25 @@ def main():
         q, kn, vn = job.q[:ns + 2].cpu(), job.kn[:ns + 2].cpu(), job.vn[:ns + 2].cpu()
         val, secs, threads, s_first, s_last = oracle_sample(wl, job.g, K, V, q0, q, kn, vn, ns, 2)
         line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle",
+                                "threads": f"numpy fp64; the Python loop over (layer, sequence) is serial, the "
+                                           f"matrix products inside it use a BLAS pool of {threads} thread(s)",
                                 "sample": f"all {wl.num_layers} layers x {wl.batch} sequence(s), decode steps "
                                           f"{s_first}-{s_last} of {wl.decode_steps} after the oracle's own prefill "
                                           f"({secs:.1f} s)"}
+        # the other LLaVA-shaped workloads, one generation each
+        if wl.name == "llava15_7b" and not args.no_others:
+            job.ctx.close()
+            del job
+            torch.cuda.empty_cache()
+            line["all_workloads"] = [other_workload_line(n, device, local)
+                                     for n in ("llava15_7b_b32", "llava15_13b_b16", "llava_next_b8")]
+            job = None
+        # oracle and GPU free-running side by side (no re-seeding): where, if anywhere, the kept sets part
+        line["free_running"] = free_running_report(wl, device)
     if rank == 0:
         print(json.dumps(line))
-    job.ctx.close()
+    if job is not None:
+        job.ctx.close()
     if dist:
         torch.distributed.destroy_process_group()
 

@@ -23,6 +23,10 @@
  *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as void*) and the call
  *     returns without waiting for it unless stated otherwise.  Calls on one context must be
  *     issued in program order; buffers must stay valid until the enqueued work has finished.
+ *   - Inputs are read in plain stream order: whatever the stream ran before the call has finished, and its
+ *     writes are visible, before a kernel of the call reads them (see st3_set_overlap for the one exception).
+ *   - A call that fails with ST3_ERR_CUDA after it has begun to enqueue work leaves the context unusable:
+ *     every later prefill or decode call on it returns ST3_ERR_BAD_STATE.  Destroy it and create a new one.
  *   - Errors are reported through the return code.  Problems detected on the device (a count
  *     that disagrees with the schedule, a non-finite score, a copy that never arrived) are
  *     OR-ed into a device status word read with st3_get_status.  The library never aborts,
@@ -133,7 +137,9 @@ st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, 
  *   text_len host [B], each in [1, max_text_len]; read before the call returns; must be the
  *                 same values for every layer range of one generation
  *   out      dev  [layer_count][B][H][D] attention output of the last prompt token
- * Resets the step counter of those layers to 0. */
+ * Resets the step counter of those layers to 0.  A call with layer_begin == 0 (or with other text lengths
+ * than the last one) opens a new generation: every other layer must be prefilled again before it decodes,
+ * so prefill layer 0 first when the layers are prefilled one call at a time. */
 st3_status st3_prefill_select(st3_ctx* ctx, int32_t layer_begin, int32_t layer_count,
                               const void* q_last, const void* k, const void* v,
                               const int32_t* text_len, void* out, void* cuda_stream);
@@ -158,6 +164,16 @@ st3_status st3_prefill_select_scored(st3_ctx* ctx, int32_t layer_begin, int32_t 
 st3_status st3_decode_step(st3_ctx* ctx, int32_t step, int32_t layer_begin, int32_t layer_count,
                            const void* q, const void* k_new, const void* v_new, void* out,
                            void* cuda_stream);
+
+/* Lets a decode step's attention kernel start while the launch ahead of it in the stream is still running
+ * (programmatic dependent launch; on = 1).  Back-to-back decode steps then overlap: the next step's attention
+ * over rows that the previous step's selection does not touch runs under that selection, and per-(layer,
+ * sequence) flags order the rest.  The price is a promise by the caller: q, k_new and v_new of a step are
+ * complete in device memory BEFORE the launch ahead of st3_decode_step in the stream begins; in particular
+ * the kernel that produces them must not signal programmatic completion (griddepcontrol.launch_dependents,
+ * cudaTriggerProgrammaticLaunchCompletion) before its last write to them.  Off by default: every kernel of
+ * a call then starts only after all earlier work of the stream has finished. */
+st3_status st3_set_overlap(st3_ctx* ctx, int32_t on);
 
 /* Same step with HOST buffers (pinned memory recommended): the library copies q/k_new/v_new to
  * staging areas inside its workspace, runs the step and copies `out` back, all on the stream.

@@ -22,7 +22,7 @@ DEV_COUNT_MISMATCH, DEV_NONFINITE, DEV_COPY_TIMEOUT, DEV_RANGE = 1, 2, 4, 8
 EXPORTS = ["st3_schedule_count", "st3_workspace_size", "st3_create", "st3_prefill_select",
            "st3_prefill_select_scored", "st3_decode_step",
            "st3_decode_step_host", "st3_get_kept", "st3_get_rows", "st3_get_status", "st3_rows_held",
-           "st3_profile_enable", "st3_profile_read", "st3_launch_count", "st3_status_string", "st3_destroy",
+           "st3_set_overlap", "st3_profile_enable", "st3_profile_read", "st3_launch_count", "st3_status_string", "st3_destroy",
            "st3_attend_noalloc", "st3_prefill_attend"]
 
 
@@ -67,6 +67,7 @@ def load():
     lib.st3_get_rows.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.st3_get_status.argtypes = [vp, C.POINTER(i32)]
     lib.st3_rows_held.argtypes = [vp, C.POINTER(i64), C.POINTER(i64)]
+    lib.st3_set_overlap.argtypes = [vp, i32]
     lib.st3_profile_enable.argtypes = [vp, i32]
     lib.st3_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(i64),
                                      C.POINTER(i64)]
@@ -159,6 +160,10 @@ def st3_rows_held(ctx):
     a, b = C.c_int64(0), C.c_int64(0)
     _check(load().st3_rows_held(ctx, C.byref(a), C.byref(b)), "st3_rows_held")
     return a.value, b.value
+
+
+def st3_set_overlap(ctx, on: bool):
+    _check(load().st3_set_overlap(ctx, int(on)), "st3_set_overlap")
 
 
 def st3_profile_enable(ctx, on: bool):

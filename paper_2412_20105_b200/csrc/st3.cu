@@ -181,6 +181,8 @@ struct st3_ctx {
   std::vector<int> logit_copy; // per layer: which copy holds the logits it wrote last
   std::vector<int> logit_step; // per layer: the step those logits belong to (-1: none)
   bool serialize_next;         // the next attention launch must wait for every earlier launch
+  bool overlap;                // st3_set_overlap: the attention launch may start before the launch ahead of it ends
+  bool failed;                 // a launch failed half-way: host bookkeeping and device state may disagree
 };
 
 namespace {
@@ -214,8 +216,10 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
   }
   (void)total_items;
   {
-    // Programmatic dependent launch: this launch may start while the previous step's finish launch is
-    // still running (that kernel allows it at its start); p.flags orders what the two share.
+    // With st3_set_overlap(ctx, 1) this is a programmatic dependent launch: it may start while the previous
+    // step's finish launch is still running (that kernel allows it at its start); p.flags orders what the two
+    // share.  The kernel reads the step's inputs without waiting for the launch ahead of it, which is only
+    // right when those inputs were complete before that launch began - hence off unless the caller says so.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(ctx->num_sms * ctx->attend_ctas_per_sm));
     cfg.blockDim = dim3(kAttendThreads);
@@ -225,7 +229,7 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = (ctx->profiling || ingest || ctx->serialize_next) ? 0 : 1;
+    cfg.numAttrs = (!ctx->overlap || ctx->profiling || ingest || ctx->serialize_next) ? 0 : 1;
     if (cudaLaunchKernelEx(&cfg, st3_attend_kernel<T, D>, p) != cudaSuccess) return ST3_ERR_CUDA;
   }
   if (e1) cudaEventRecord(e1, st);
@@ -358,7 +362,12 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
 #define ST3_LAUNCH(T, D) launch_step_t<T, D>(ctx, p, (int)total_items, st, k, v, prefill, ext_scores ? &psel : nullptr)
   const st3_status s = ST3_DISPATCH(ctx, ST3_LAUNCH);
 #undef ST3_LAUNCH
-  if (s != ST3_OK) return s;
+  if (s != ST3_OK) {
+    // Some kernel of the call may already be enqueued (the device work counter, the flags and the cache then
+    // move on without the host's bookkeeping): nothing later on this context can be trusted.
+    ctx->failed = true;
+    return s;
+  }
   for (int i = 0; i < layer_count; ++i) {
     ctx->n_host[layer_begin + i] = p.ntgt[i];
     ctx->last_step[layer_begin + i] = step;
@@ -423,6 +432,8 @@ st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, 
   ctx->logit_copy.assign(cfg->num_layers, 0);
   ctx->logit_step.assign(cfg->num_layers, -1);
   ctx->serialize_next = false;
+  ctx->overlap = false;
+  ctx->failed = false;
   ctx->profiling = false;
   ctx->ev_used = 0;
   ctx->attend_smem = kSlots * (2 * tile_bytes(cfg) + kQBytes);
@@ -454,6 +465,7 @@ static st3_status prefill_common(st3_ctx* ctx, int32_t layer_begin, int32_t laye
                                  const void* k, const void* v, const int32_t* text_len, const float* scores,
                                  void* out, void* cuda_stream) {
   if (!ctx || !text_len) return ST3_ERR_INVALID_ARG;
+  if (ctx->failed) return ST3_ERR_BAD_STATE;
   const st3_config& c = ctx->cfg;
   if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c.num_layers) return ST3_ERR_INVALID_ARG;
   if (!aligned16(q_last) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return ST3_ERR_INVALID_ARG;
@@ -464,14 +476,16 @@ static st3_status prefill_common(st3_ctx* ctx, int32_t layer_begin, int32_t laye
     mx = text_len[b] > mx ? text_len[b] : mx;
   }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  bool changed = !ctx->have_text;
-  for (int b = 0; b < c.batch && !changed; ++b) changed = ctx->text_len[b] != text_len[b];
-  if (changed) {
-    // a new generation: every layer must be prefilled again before it can decode
+  // A call that starts at layer 0, or that brings other text lengths, opens a new generation: every layer
+  // must be prefilled again before it can decode.
+  bool differs = !ctx->have_text;
+  for (int b = 0; b < c.batch && !differs; ++b) differs = ctx->text_len[b] != text_len[b];
+  if (differs || layer_begin == 0)
+    for (int l = 0; l < c.num_layers; ++l) { ctx->last_step[l] = -1; ctx->logit_step[l] = -1; }
+  if (differs) {
     for (int b = 0; b < c.batch; ++b) ctx->text_len[b] = text_len[b];
     ctx->max_text = mx;
     ctx->have_text = true;
-    for (int l = 0; l < c.num_layers; ++l) ctx->last_step[l] = -1;
     // pageable source: the runtime stages it before returning, so ctx->text_len may change later
     if (cudaMemcpyAsync(ctx->ws + ctx->lay.text_len, ctx->text_len.data(), (size_t)c.batch * sizeof(int),
                         cudaMemcpyHostToDevice, st) != cudaSuccess)
@@ -496,6 +510,7 @@ st3_status st3_prefill_select_scored(st3_ctx* ctx, int32_t layer_begin, int32_t 
 st3_status st3_decode_step(st3_ctx* ctx, int32_t step, int32_t layer_begin, int32_t layer_count, const void* q,
                            const void* k_new, const void* v_new, void* out, void* cuda_stream) {
   if (!ctx) return ST3_ERR_INVALID_ARG;
+  if (ctx->failed) return ST3_ERR_BAD_STATE;
   const st3_config& c = ctx->cfg;
   if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c.num_layers) return ST3_ERR_INVALID_ARG;
   if (step < 1) return ST3_ERR_INVALID_ARG;
@@ -601,6 +616,12 @@ st3_status st3_rows_held(st3_ctx* ctx, int64_t* visual_rows, int64_t* other_rows
   }
   if (visual_rows) *visual_rows = vis;
   if (other_rows) *other_rows = oth;
+  return ST3_OK;
+}
+
+st3_status st3_set_overlap(st3_ctx* ctx, int32_t on) {
+  if (!ctx) return ST3_ERR_INVALID_ARG;
+  ctx->overlap = on != 0;
   return ST3_OK;
 }
 

@@ -35,11 +35,13 @@ constexpr int kKBoxBytes = kKeys * 128;  // one TMA box of K or V: 64 rows x 64 
 constexpr int kKTileBytes = 2 * kKBoxBytes;
 constexpr uint32_t kTmemCols = 256;   // S in columns [0,64), O in [128,256)
 
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+// One box of [rows][64 bf16] of instance z, starting at row y (may be negative or reach past the instance's
+// last row: such rows are filled with zeros, never with a neighbouring instance's data) and column x (0 or 64).
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int x, int y, int z, uint64_t* bar) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(
           smem_u32(dst)),
-      "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+      "l"(map), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar))
       : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_cta(uint64_t* bar) {
@@ -202,7 +204,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   const int row_base = inst * T;  // first row of this instance in the [num_inst * T][128] tensors
   // Query tiles are aligned to the END of the prompt: the ragged tile is the first one, where the causal prefix
   // is shortest, instead of the last one, where a mostly empty tile would walk every key.  Its rows before the
-  // prompt (q0 < 0) are dead: their loads read the fill value or a neighbour's rows, nothing is stored.
+  // prompt (q0 < 0) are dead: their loads read the fill value (zeros), nothing is stored.
   const int q0 = T - ((int)gridDim.x - qt) * kTile;                // first query row of this tile
   const int nkt = (q0 + kTile + kKeys - 1) / kKeys;                // causal: key tiles up to the diagonal
 
@@ -214,19 +216,19 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     s_fail = 0;
     mbar_fence_init();
     mbar_expect_tx(&bar_q, kTileBytes2);
-    tma_load_2d(sQ, &map_q, 0, row_base + q0, &bar_q);
-    tma_load_2d(sQ + kBoxBytes, &map_q, 64, row_base + q0, &bar_q);
+    tma_load_3d(sQ, &map_q, 0, q0, inst, &bar_q);
+    tma_load_3d(sQ + kBoxBytes, &map_q, 64, q0, inst, &bar_q);
     for (int kt = 0; kt < 3 && kt < nkt; ++kt) {
       unsigned char* d = sK2 + kt * kKTileBytes;
       mbar_expect_tx(&bar_k[kt], kKTileBytes);
-      tma_load_2d(d, &map_k, 0, row_base + kt * kKeys, &bar_k[kt]);
-      tma_load_2d(d + kKBoxBytes, &map_k, 64, row_base + kt * kKeys, &bar_k[kt]);
+      tma_load_3d(d, &map_k, 0, kt * kKeys, inst, &bar_k[kt]);
+      tma_load_3d(d + kKBoxBytes, &map_k, 64, kt * kKeys, inst, &bar_k[kt]);
     }
     for (int kt = 0; kt < 2 && kt < nkt; ++kt) {
       unsigned char* d = sV2 + kt * kKTileBytes;
       mbar_expect_tx(&bar_v[kt], kKTileBytes);
-      tma_load_2d(d, &map_v, 0, row_base + kt * kKeys, &bar_v[kt]);
-      tma_load_2d(d + kKBoxBytes, &map_v, 64, row_base + kt * kKeys, &bar_v[kt]);
+      tma_load_3d(d, &map_v, 0, kt * kKeys, inst, &bar_v[kt]);
+      tma_load_3d(d + kKBoxBytes, &map_v, 64, kt * kKeys, inst, &bar_v[kt]);
     }
   }
   __syncthreads();
@@ -250,14 +252,14 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
     auto load_k = [&](int kt) {
       unsigned char* d = sK2 + (kt % 3) * kKTileBytes;
       mbar_expect_tx(&bar_k[kt % 3], kKTileBytes);
-      tma_load_2d(d, &map_k, 0, row_base + kt * kKeys, &bar_k[kt % 3]);
-      tma_load_2d(d + kKBoxBytes, &map_k, 64, row_base + kt * kKeys, &bar_k[kt % 3]);
+      tma_load_3d(d, &map_k, 0, kt * kKeys, inst, &bar_k[kt % 3]);
+      tma_load_3d(d + kKBoxBytes, &map_k, 64, kt * kKeys, inst, &bar_k[kt % 3]);
     };
     auto load_v = [&](int kt) {
       unsigned char* d = sV2 + (kt & 1) * kKTileBytes;
       mbar_expect_tx(&bar_v[kt & 1], kKTileBytes);
-      tma_load_2d(d, &map_v, 0, row_base + kt * kKeys, &bar_v[kt & 1]);
-      tma_load_2d(d + kKBoxBytes, &map_v, 64, row_base + kt * kKeys, &bar_v[kt & 1]);
+      tma_load_3d(d, &map_v, 0, kt * kKeys, inst, &bar_v[kt & 1]);
+      tma_load_3d(d + kKBoxBytes, &map_v, 64, kt * kKeys, inst, &bar_v[kt & 1]);
     };
     // S(kt) = Q K(kt)^T: 8 steps of 16 along the head dimension
     const uint32_t q_lo = desc_lo(smem_u32(sQ), 16), k_lo = desc_lo(smem_u32(sK2), 16);
@@ -468,13 +470,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// [rows][128] bf16 tensor, boxes of box_rows rows x 64 columns, 128-byte swizzle, out-of-range rows read as zero.
-bool make_map(EncodeTiledFn fn, CUtensorMap* map, const void* base, size_t rows, int box_rows) {
-  const cuuint64_t dims[2] = {128, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {256};
-  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+// [num_inst][rows][128] bf16 tensor, boxes of box_rows rows x 64 columns inside one instance, 128-byte swizzle;
+// rows outside [0, rows) of the instance read as zero, so a tile at the end of one instance never sees the next.
+bool make_map(EncodeTiledFn fn, CUtensorMap* map, const void* base, size_t num_inst, size_t rows, int box_rows) {
+  const cuuint64_t dims[3] = {128, (cuuint64_t)rows, (cuuint64_t)num_inst};
+  const cuuint64_t strides[2] = {256, (cuuint64_t)rows * 256};
+  const cuuint32_t box[3] = {64, (cuuint32_t)box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -503,9 +506,9 @@ extern "C" st3_status st3_prefill_attend(const void* q, const void* k, const voi
   }();
   if (!encode) return ST3_ERR_CUDA;
   CUtensorMap mq, mk, mv;
-  const size_t rows = (size_t)num_inst * seq_len;
-  if (!make_map(encode, &mq, q, rows, kTile) || !make_map(encode, &mk, k, rows, kKeys) ||
-      !make_map(encode, &mv, v, rows, kKeys))
+  if (!make_map(encode, &mq, q, (size_t)num_inst, (size_t)seq_len, kTile) ||
+      !make_map(encode, &mk, k, (size_t)num_inst, (size_t)seq_len, kKeys) ||
+      !make_map(encode, &mv, v, (size_t)num_inst, (size_t)seq_len, kKeys))
     return ST3_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const int smem = kPfSmem;

@@ -43,12 +43,17 @@ def assert_rank_ordered(ref_mass, got_ids, where="", rel=1e-3):
 
 
 class GpuRun:
-    def __init__(self, wl: Workload, device="cuda:0", sched_kw=None, **cfg_overrides):
+    def __init__(self, wl: Workload, device="cuda:0", sched_kw=None, overlap=False, **cfg_overrides):
+        """`overlap`: back-to-back steps overlap on the GPU (st3_set_overlap); the inputs of a step are then
+        generated and synchronised before the step is enqueued, as that mode requires."""
         self.wl, self.dev = wl, torch.device(device)
         self.g = SynthInputs(wl)
         self.sched = make_schedule(wl, disable_trim=bool(cfg_overrides.get("disable_trim", 0)), **(sched_kw or {}))
         self.cfg = B.config_from_workload(wl, **cfg_overrides)
         self.ctx = B.Context(self.cfg, device)
+        self.overlap = bool(overlap)
+        self._ahead = {}
+        B.st3_set_overlap(self.ctx.handle, self.overlap)
         self.L = wl.num_layers
         self.out = torch.empty(self.ctx.io_shape(), dtype=self.ctx.dtype, device=self.dev)
         self.stats = {"exact": 0, "near-tie": 0, "units": 0}
@@ -106,6 +111,16 @@ class GpuRun:
 
     def inputs(self, step):
         g = self.g
+        if self.overlap:
+            # steps that overlap need their inputs complete before the launch ahead of them begins: generate a
+            # block of steps, wait for it, then hand the steps out one by one
+            if step not in self._ahead:
+                steps = list(range(step, min(self.wl.decode_steps, step + 15) + 1))
+                q = g.queries(steps, device=self.dev)
+                kn, vn = g.new_kv(steps, device=self.dev)
+                torch.cuda.synchronize(self.dev)
+                self._ahead = {t: (q[i], kn[i], vn[i]) for i, t in enumerate(steps)}
+            return self._ahead[step]
         q = g.queries([step], device=self.dev)[0]
         kn, vn = g.new_kv([step], device=self.dev)
         return q, kn[0], vn[0]

@@ -233,3 +233,61 @@ def test_two_score_levels_with_ties_at_the_cut():
         assert ctx.status() == 0
     finally:
         ctx.close()
+
+
+def test_inputs_from_a_producer_that_signals_completion_early():
+    """q, k_new and v_new of every step are written by a kernel that allows its dependents to launch and only
+    then, 30 us later, writes them.  In the default mode the step must still see the written values (its
+    kernels start only when the producer's grid has finished): the outputs equal those of a run whose inputs
+    were in place long before."""
+    import native
+    lib = native.load()
+    wl = _small()
+    a, b = GpuRun(wl), GpuRun(wl)
+    try:
+        a.prefill(); b.prefill()
+        st = torch.cuda.current_stream().cuda_stream
+        for t in range(1, 6):
+            a.decode(t)
+            q, kn, vn = b.inputs(t)
+            src = torch.stack([q, kn, vn]).contiguous()
+            dst = torch.zeros_like(src)                         # stale contents: zeros
+            torch.cuda.synchronize()
+            n16 = src.numel() * src.element_size() // 16
+            assert lib.st3_test_early_trigger_copy(dst.data_ptr(), src.data_ptr(), n16, 30, st) == 0
+            b.ctx.decode_step(t, dst[0], dst[1], dst[2], b.out)
+            torch.cuda.synchronize()
+            assert torch.equal(a.out, b.out), t
+            for l in range(wl.num_layers):
+                ia, ca, _ = a.kept(l)
+                ib, cb, _ = b.kept(l)
+                assert np.array_equal(ca, cb) and all(np.array_equal(ia[s, :ca[s]], ib[s, :cb[s]])
+                                                      for s in range(wl.batch))
+            b.check_rows_unit(0, 1, 0, t)                       # the appended rows are the written ones too
+        assert a.ctx.status() == 0 and b.ctx.status() == 0
+    finally:
+        a.close(); b.close()
+
+
+def test_a_new_generation_starts_at_layer_zero():
+    """Prefilling layer 0 opens a new generation: layers that have not been prefilled again cannot decode."""
+    wl = _small()
+    run = GpuRun(wl)
+    try:
+        run.prefill()
+        run.decode(1)
+        g = run.g
+        q0 = g.queries([0], device=run.dev)[0]
+        K, V = g.prompt_kv([0, 1], device=run.dev)
+        run.ctx.prefill_select(q0[0:2].contiguous(), K, V, g.text_len.tolist(), run.out[0:2], layer_begin=0)
+        q, kn, vn = run.inputs(1)
+        run.ctx.decode_step(1, q[0:2], kn[0:2], vn[0:2], run.out[0:2], layer_begin=0)     # prefilled again: fine
+        with pytest.raises(B.St3Error) as e:                                              # layers 2.. are stale
+            run.ctx.decode_step(1, q[2:], kn[2:], vn[2:], run.out[2:], layer_begin=2)
+        assert e.value.code == 3
+        with pytest.raises(B.St3Error) as e:
+            run.ctx.decode_step(2, q[2:], kn[2:], vn[2:], run.out[2:], layer_begin=2)
+        assert e.value.code == 3
+        assert run.ctx.status() == 0
+    finally:
+        run.close()

@@ -18,10 +18,10 @@ def test_generator_is_bit_identical_on_cpu_and_gpu():
     assert torch.equal(g.queries([0, 5], [7]), g.queries([0, 5], [7], device="cuda:0").cpu())
 
 
-@pytest.mark.parametrize("tau", [50.0, 10.0])
-def test_tiny_every_step(tau):
+@pytest.mark.parametrize("tau,overlap", [(50.0, False), (10.0, False), (50.0, True)])
+def test_tiny_every_step(tau, overlap):
     wl = get_workload("tiny").scaled(tau=tau)
-    stats = run_and_check(wl, wl.decode_steps)
+    stats = run_and_check(wl, wl.decode_steps, overlap=overlap)
     assert stats["units"] == wl.decode_steps + 1
 
 
@@ -44,6 +44,7 @@ def test_small_odd_shapes(dtype, D, H):
                                      first_prune_layer=1, stride=2, step_ratio_bp=2000, tau=9.0, num_planted=7)
     run_and_check(wl, 9)
     run_and_check(wl, 5, layers_per_call=2)
+    run_and_check(wl, 9, layers_per_call=2, overlap=True)
 
 
 def test_largest_visual_span_and_head_count():
@@ -72,10 +73,12 @@ def test_llava15_7b_first_steps_all_units():
     assert stats["units"] == 32 * 4
 
 
-def test_llava15_7b_full_length_sampled_steps():
+@pytest.mark.parametrize("overlap", [False, True])
+def test_llava15_7b_full_length_sampled_steps(overlap):
+    """`overlap`: consecutive steps overlap on the GPU (the mode bench.py times) or run in plain stream order."""
     wl = get_workload("llava15_7b")
     steps = [0, 1, 2, 17, 64, 128, 129, 200, 254, 255, 256]
-    stats = run_and_check(wl, wl.decode_steps, check_steps=steps)
+    stats = run_and_check(wl, wl.decode_steps, check_steps=steps, overlap=overlap)
     assert stats["units"] == 32 * len(steps)
 
 
@@ -85,14 +88,32 @@ def _sampled_units(wl, n, seed):
     return [(int(r.integers(wl.batch)), int(l)) for l in layers]
 
 
+def _covering_units(wl, n, seed):
+    """At least n distinct (sequence, layer) units: every pruning layer (stage head), the first and the last
+    layer, the sequences with the shortest and the longest text, the rest drawn at random."""
+    r = np.random.default_rng(seed)
+    text = SynthInputs(wl).text_len
+    b_short, b_long = int(np.argmin(text)), int(np.argmax(text))
+    heads = list(range(wl.first_prune_layer, wl.num_layers, wl.stride))
+    units = {(b_short, 0), (b_long, wl.num_layers - 1), (b_long, 1), (b_short, wl.num_layers - 1)}
+    for i, l in enumerate(heads):
+        units.add(((b_short, b_long)[i % 2], l))
+        units.add((int(r.integers(wl.batch)), l))
+    while len(units) < n:
+        units.add((int(r.integers(wl.batch)), int(r.integers(wl.num_layers))))
+    return sorted(units, key=lambda u: (u[1], u[0]))
+
+
 @pytest.mark.parametrize("name,steps", [("llava15_7b_b32", [0, 1, 100, 300, 511, 512]),
-                                        ("llava15_13b_b16", [0, 1, 256, 512]),
+                                        ("llava15_13b_b16", [0, 1, 256, 511, 512]),
                                         ("llava_next_b8", [0, 1, 500, 1023, 1024])])
 def test_full_size_workloads_sampled_units(name, steps):
+    """The batched workloads at full size and full length, launched as bench.py launches them (all layers per
+    call, steps overlapping): 32 or more units, every pruning layer among them, are judged at the sampled steps."""
     wl = get_workload(name)
-    units = _sampled_units(wl, 5, wl.seed)
-    lpc = 8 if wl.batch > 1 else None
-    stats = run_and_check(wl, wl.decode_steps, check_steps=steps, units=units, layers_per_call=None, rows_checks=1)
+    units = _covering_units(wl, 32, wl.seed)
+    assert len(units) >= 32
+    stats = run_and_check(wl, wl.decode_steps, check_steps=steps, units=units, rows_checks=2, overlap=True)
     assert stats["units"] == len(units) * len(steps)
 
 
@@ -197,3 +218,20 @@ def test_stage_shared_13b_sampled():
     units = sorted(set(units) | set(heads), key=lambda u: (u[1], u[0]))
     stats = run_and_check(wl, 40, check_steps=[0, 1, 20, 40], units=units, rows_checks=1, stage_shared=1)
     assert stats["units"] == len(units) * 4
+
+
+@pytest.mark.parametrize("name", ["tiny", "llava15_7b"])
+def test_free_running_against_the_oracle(name):
+    """Oracle and GPU run a whole generation without either adopting the other's state.  Where the kept sets
+    part (if they do) the oracle's scores at that cut must be a near-tie; until then outputs stay in tolerance."""
+    import bench
+    from gpu_harness import OUT_ABS_F32, OUT_REL_BF16
+    wl = get_workload(name)
+    rep = bench.free_running_report(wl, torch.device("cuda:0"))
+    print("free-running:", rep)
+    assert rep["steps_compared"] == wl.decode_steps and rep["units"] == wl.num_layers * wl.batch
+    first = rep["first_divergence"]
+    assert first is None or first["near_tie"], first
+    if first is None:
+        assert rep["units_diverged_by_the_end"] == 0
+    assert rep["max_output_error_while_in_agreement"] <= (OUT_ABS_F32 if wl.dtype == "f32" else OUT_REL_BF16)

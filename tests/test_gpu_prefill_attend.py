@@ -10,12 +10,14 @@ from paper_2412_20105_b200.build import build
 pytestmark = pytest.mark.gpu
 
 
-def _run(T, H, nb, sys_len, nv, seed):
+def _run(T, H, nb, sys_len, nv, seed, poison=None):
     build()
     g = torch.Generator().manual_seed(seed)
     n = nb * H
     mk = lambda: torch.randn(n, T, 128, generator=g).to(torch.bfloat16).cuda()
     q, k, v = mk(), mk(), mk()
+    if poison is not None:
+        poison(q, k, v)
     out = torch.full((n, T, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
     probs = torch.zeros(n, max(1, nv), device="cuda")
     scores = torch.zeros(nb, max(1, nv), device="cuda")
@@ -44,6 +46,28 @@ def test_causal_attention_and_next_layer_scores(T, H, nb, sys_len, nv):
         assert excess.max() <= 0, f"causal out b={b}: error exceeds the bf16 bound by {excess.max()}"
         want = A[:, T - 1, sys_len:sys_len + nv].sum(axis=0)            # alpha: last row, visual slice, over heads
         assert np.allclose(scores[b, :nv].cpu().numpy(), want, rtol=2e-3, atol=1e-7)
+
+
+@pytest.mark.parametrize("T", [37, 100, 131])
+def test_tiles_never_read_the_neighbouring_instance(T):
+    """T is not a multiple of the 64-key tile: the last key tile of an instance reaches past its end.  The rows
+    it would find there in a flat layout are the NEXT instance's first rows; they hold Inf/NaN here.  Keys past
+    the end carry probability 0, and 0 x Inf = NaN would poison the output if those rows were ever loaded; rows
+    outside the instance must read as zeros instead."""
+    H, nb, sys_len, nv = 2, 2, 3, 20
+
+    def poison(q, k, v):
+        # the first rows of every instance but the first (what the previous instance's last tile overhangs)
+        v[1:, :64] = float("inf")
+        k[1:, :64] = float("nan")
+        q[1:, :64] = float("nan")
+
+    q, k, v, out, scores = _run(T, H, nb, sys_len, nv, seed=T, poison=poison)
+    ref, A = O.causal_attention(q[:1].double().cpu().numpy(), k[:1].double().cpu().numpy(), v[:1].double().cpu().numpy())
+    got = out[0].double().cpu().numpy()                  # instance 0 is clean; its neighbour is poisoned
+    assert np.all(np.isfinite(got))
+    bound = 2.0 ** -8 * (np.matmul(A, np.abs(v[:1].double().cpu().numpy())) + np.abs(ref)) + 1e-6
+    assert (np.abs(got - ref[0]) - bound[0]).max() <= 0
 
 
 def test_full_prompt_length_sampled_rows():

@@ -41,19 +41,39 @@ def _inputs(seed, H, T, D, dtype):
     return mk(H, D) * 2.0, mk(H, T, D), mk(H, T, D)
 
 
+# every kernel instance (element type x head size), with row counts that make one chunk, a chunk boundary, a
+# ragged last chunk of a single row, and a single-row input
+CASES = [(32, 675, 128, "bf16"), (8, 200, 64, "f32"), (5, 129, 64, "bf16"), (3, 127, 128, "f32"),
+         (4, 1, 128, "f32"), (2, 1, 64, "bf16"), (7, 128, 64, "bf16"), (6, 257, 128, "bf16")]
+
+
+def _check_call(seed, H, T, D, dtype, stream):
+    q, k, v = _inputs(seed, H, T, D, dtype)
+    out = torch.empty_like(q)
+    B.st3_attend_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), H, T, D, dtype, stream)
+    torch.cuda.synchronize()
+    ref = _regular(q, k, v, dtype)
+    assert_out_close(f64(out), f64(ref), dtype, f"noalloc call {seed}")
+    # and both agree with plain softmax attention in fp64
+    p = torch.softmax(torch.einsum("htd,hd->ht", k.double(), q.double()) / D ** 0.5, dim=1)
+    assert_out_close(f64(out), f64(torch.einsum("ht,htd->hd", p, v.double())), dtype, f"noalloc vs fp64 {seed}")
+
+
 def test_two_calls_in_a_row_match_the_workspace_path():
     build()
     stream = torch.cuda.current_stream().cuda_stream
-    for seed, (H, T, D, dtype) in enumerate([(32, 675, 128, "bf16"), (8, 200, 64, "f32")]):
-        q, k, v = _inputs(seed, H, T, D, dtype)
-        out = torch.empty_like(q)
-        B.st3_attend_noalloc(q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), H, T, D, dtype, stream)
-        torch.cuda.synchronize()
-        ref = _regular(q, k, v, dtype)
-        assert_out_close(f64(out), f64(ref), dtype, f"noalloc call {seed}")
-        # and both agree with plain softmax attention in fp64
-        p = torch.softmax(torch.einsum("htd,hd->ht", k.double(), q.double()) / D ** 0.5, dim=1)
-        assert_out_close(f64(out), f64(torch.einsum("ht,htd->hd", p, v.double())), dtype, f"noalloc vs fp64 {seed}")
+    for seed, (H, T, D, dtype) in enumerate(CASES[:2]):
+        _check_call(seed, H, T, D, dtype, stream)
+
+
+@pytest.mark.parametrize("first,second", [(0, 2), (2, 3), (3, 4), (1, 5), (6, 7), (7, 0)])
+def test_every_kernel_instance_and_ragged_row_counts(first, second):
+    """Two calls in a row again, over all four (element type, head size) instances and the chunk edge cases;
+    the second call runs on whatever partials the first one left in the shared array."""
+    build()
+    stream = torch.cuda.current_stream().cuda_stream
+    for i in (first, second):
+        _check_call(100 + i, *CASES[i], stream)
 
 
 def test_sizes_beyond_the_static_array_are_rejected():

@@ -125,24 +125,48 @@ class ClockSampler:
 # ----------------------------------------------------------------------------------------------
 # algorithmic bytes of the attention kernel
 # ----------------------------------------------------------------------------------------------
+FOLLOWERS_PER_ITEM = 62  # lazy layers whose values ride on one work item of their source (kMaxFollow in the kernels)
+
+
+def lazy_offsets(cfg):
+    """{layer: k} for every lazy layer: it is the k-th lazy layer above its source (QK heredity, Eq. 6)."""
+    out, k = {}, 0
+    for l in range(cfg.num_layers):
+        k = k + 1 if (cfg.lazy_mask >> l) & 1 else 0
+        if k:
+            out[l] = k
+    return out
+
+
 def attend_bytes(wl, cfg, B_mod, text_len, step):
     """Bytes the attention kernel of one launch must move (all layers, all sequences).
 
     Per (sequence, layer): every cached K and V row once (r*T_cur, the newest row read from the
     step's inputs), the newest row written to the cache (r), the query (H*D*e) and, where the
-    layer evicts at this step, one fp32 logit per head per visual row (4*H*n_cur).
+    layer evicts at this step, one fp32 logit per head per visual row (4*H*n_cur).  A lazy layer
+    (QK heredity) whose values ride on its source's work items moves its V rows only (r/2 per row,
+    no query).
     """
     e = 2 if wl.dtype == "bf16" else 4
     H, D = wl.num_heads, wl.head_dim
     r = 2 * H * D * e
+    lazy = lazy_offsets(cfg)
+    pruning = lambda l: l if not cfg.stage_shared or l < wl.first_prune_layer else \
+        wl.first_prune_layer + (l - wl.first_prune_layer) // wl.stride * wl.stride
     total = 0
     for l in range(wl.num_layers):
         n_cur = wl.num_visual if step == 0 else B_mod.st3_schedule_count(cfg, l, step - 1)
         n_tgt = B_mod.st3_schedule_count(cfg, l, step)
+        rides = l in lazy and lazy[l] % (FOLLOWERS_PER_ITEM + 1) != 0
         for b in range(wl.batch):
             t_cur = wl.sys_len + n_cur + int(text_len[b]) + step
-            total += r * t_cur + (r if step > 0 else 0) + H * D * e
-            if n_tgt < n_cur:
+            if rides:
+                total += (r // 2) * t_cur + (r // 2 if step > 0 else 0)
+            elif l in lazy:
+                total += r * t_cur + (r // 2 if step > 0 else 0) + H * D * e
+            else:
+                total += r * t_cur + (r if step > 0 else 0) + H * D * e
+            if n_tgt < n_cur and pruning(l) == l:
                 total += 4 * H * n_cur
     return total
 
@@ -159,16 +183,19 @@ def path_bytes(wl, cfg, B_mod, text_len):
     e = 2 if wl.dtype == "bf16" else 4
     H, D = wl.num_heads, wl.head_dim
     r = 2 * H * D * e
+    lazy = lazy_offsets(cfg)
     total = 0
     for step in range(0, wl.decode_steps + 1):
         for l in range(wl.num_layers):
             n_cur = wl.num_visual if step == 0 else B_mod.st3_schedule_count(cfg, l, step - 1)
             n_tgt = min(n_cur, B_mod.st3_schedule_count(cfg, l, step))
+            # a lazy layer has no keys and no query of its own (Eq. 6): half the row bytes, output only
+            rl, io = (r // 2, H * D * e) if l in lazy else (r, 2 * H * D * e)
             for b in range(wl.batch):
                 t_cur = wl.sys_len + n_cur + int(text_len[b]) + step
-                total += r * t_cur + 2 * H * D * e + (2 * r if step > 0 else 2 * r * t_cur)
+                total += rl * t_cur + io + (2 * rl if step > 0 else 2 * rl * t_cur)
                 if n_tgt < n_cur:
-                    total += (8 * H + 8) * n_cur + 2 * r * (n_cur - n_tgt)
+                    total += (8 * H + 8) * n_cur + 2 * rl * (n_cur - n_tgt)
     return total
 
 
@@ -192,7 +219,8 @@ def f64(t):
 class Job:
     """All device-resident inputs of one workload plus a library context."""
 
-    def __init__(self, wl, device, disable_trim=False, rows_per_chunk=0, static_rank=False):
+    def __init__(self, wl, device, disable_trim=False, rows_per_chunk=0, static_rank=False, stage_shared=False,
+                 lazy_mask=0, host_prefill=False):
         from paper_2412_20105_b200 import binding as B
         from paper_2412_20105_b200.build import build
         build()
@@ -200,7 +228,8 @@ class Job:
         self.wl, self.dev = wl, device
         self.g = SynthInputs(wl)
         self.cfg = B.config_from_workload(wl, disable_trim=int(disable_trim), rows_per_chunk=rows_per_chunk,
-                                           static_rank=int(static_rank))
+                                           static_rank=int(static_rank), stage_shared=int(stage_shared),
+                                           lazy_mask=int(lazy_mask), host_prefill=int(host_prefill))
         self.ctx = B.Context(self.cfg, device)
         # every input of a generation is in device memory before its first launch, which is what the
         # overlapping-steps mode asks of its caller
@@ -316,6 +345,7 @@ class Job:
         return out
 
     def make_host(self):
+        """Every input of a generation in pinned host memory, and pinned buffers for every output."""
         self.hK, self.hV = self.K.cpu().pin_memory(), self.V.cpu().pin_memory()
         self.hq0 = self.q0.cpu().pin_memory()
         # one pinned buffer [step][q | k_new | v_new]: the three inputs of a step lie back to back, which lets the
@@ -324,17 +354,13 @@ class Job:
         self.hq = self.hqkv[:, 0]
         self.hout = torch.empty_like(self.hq).pin_memory()
         self.hout0 = torch.empty_like(self.hq0).pin_memory()
-        self.dK, self.dV, self.dq0 = torch.empty_like(self.K), torch.empty_like(self.V), torch.empty_like(self.q0)
 
     def generation_host(self):
-        """Same work, every input starting in pinned host memory and every output ending there."""
+        """Same work through the host-buffer calls of the C ABI: every input starts in pinned host memory and
+        every output ends there (the context was created with host_prefill = 1)."""
         B, h, L, st = self.B, self.ctx.handle, self.wl.num_layers, self.stream
-        self.dK.copy_(self.hK, non_blocking=True)
-        self.dV.copy_(self.hV, non_blocking=True)
-        self.dq0.copy_(self.hq0, non_blocking=True)
-        B.st3_prefill_select(h, 0, L, self.dq0.data_ptr(), self.dK.data_ptr(), self.dV.data_ptr(), self.text,
-                             self.out0.data_ptr(), st)
-        self.hout0.copy_(self.out0, non_blocking=True)
+        B.st3_prefill_select_host(h, 0, L, self.hq0.data_ptr(), self.hK.data_ptr(), self.hV.data_ptr(), self.text,
+                                  self.hout0.data_ptr(), st)
         base, o, nb = self.hqkv.data_ptr(), self.hout.data_ptr(), self.io_bytes
         step_fn = self.lib.st3_decode_step_host
         for t in range(1, self.wl.decode_steps + 1):
@@ -343,6 +369,7 @@ class Job:
             rc = step_fn(h, t, 0, L, q, q + nb, q + 2 * nb, o + off, st)
             if rc:
                 raise B.St3Error(rc, f"st3_decode_step_host t={t}")
+        B.st3_host_sync(h, st)
 
     def h2d_bytes(self):
         kv = 2 * self.K.numel() * self.K.element_size()
@@ -569,6 +596,25 @@ def add_path_fraction(roofline, job, ms_per_generation):
     return roofline
 
 
+def qk_heredity_line(wl, device, args, name, mask):
+    """One configuration with stage-shared kept sets and the given lazy layers: tokens/s, the attention
+    kernel's algorithmic bytes per launch (lazy layers count their V rows only) and its fraction of the peak."""
+    job = Job(wl, device, stage_shared=True, lazy_mask=mask, rows_per_chunk=args.rows_per_chunk)
+    try:
+        for _ in range(3):
+            job.generation()
+        ms = timed(job.generation, args.steps, False)
+        job.ctx.status()
+        roof = kernel_roofline(job, 1, 1)
+        return {"lazy_layers": name, "value": wl.batch * wl.decode_steps * args.steps / (ms * 1e-3), "unit": UNIT,
+                "algorithmic_bytes_per_launch": roof["algorithmic_bytes_per_launch"],
+                "us_per_launch": roof["us_per_launch"], "frac": roof["frac"]}
+    finally:
+        job.ctx.close()
+        del job
+        torch.cuda.empty_cache()
+
+
 def other_workload_line(name, device, rank):
     """One timed generation of another LLaVA-shaped workload (after one warm-up generation): tokens/s, the
     attention kernel's and the whole path's fraction of the HBM peak, clocks during the timed generation."""
@@ -602,9 +648,14 @@ def main():
     ap.add_argument("--workload", default="llava15_7b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows-per-chunk", type=int, default=0)
+    ap.add_argument("--stage-shared", action="store_true",
+                    help="layers between two pruning layers keep the pruning layer's tokens (strided pruning)")
+    ap.add_argument("--lazy-mask", type=lambda x: int(x, 0), default=0,
+                    help="bit l set: layer l is lazy (QK heredity); needs --stage-shared inside a pruning stage")
     ap.add_argument("--no-extras", action="store_true", help="skip the e2e, unpruned and cpu_baseline legs")
+    ap.add_argument("--e2e-only", action="store_true", help="after the timed run, only the end-to-end leg")
     ap.add_argument("--no-others", action="store_true", help="skip the one-generation runs of the other workloads")
-    ap.add_argument("--leg", default="", choices=["", "prefill_attend"],
+    ap.add_argument("--leg", default="", choices=["", "prefill_attend", "qk_heredity"],
                     help="run one auxiliary leg alone and print its JSON (for timing or profiling that kernel)")
     ap.add_argument("--instances", type=int, default=2048, help="cap on the (sequence, head) instances of --leg")
     args = ap.parse_args()
@@ -661,10 +712,19 @@ def main():
             print(json.dumps({"leg": args.leg, "workload": wl.name,
                               **(prefill_attend_leg(wl, device, max(1, args.steps), args.instances) or {})}))
         return
+    if args.leg == "qk_heredity":
+        if rank == 0:
+            print(json.dumps({"leg": args.leg, "workload": wl.name, "lines": [
+                qk_heredity_line(wl, device, args, name, mask) for name, mask in (
+                    ("stage_shared, no lazy layer", 0), ("layers 29-30 inherit layer 28", (1 << 29) | (1 << 30)),
+                    ("layers 4-6 inherit layer 3, layers 8-9 inherit layer 7", sum(1 << l for l in (4, 5, 6, 8, 9))))]}))
+        return
     if dist:
         torch.distributed.init_process_group("nccl", device_id=device)
     wl = replica_workload(wl, rank, world)
-    job = Job(wl, device, rows_per_chunk=args.rows_per_chunk)
+    job = Job(wl, device, rows_per_chunk=args.rows_per_chunk, stage_shared=args.stage_shared, lazy_mask=args.lazy_mask)
+    if args.stage_shared or args.lazy_mask:
+        config["variant"] = f"stage_shared={int(args.stage_shared)} lazy_mask={args.lazy_mask:#x}"
     B = job.B
     tokens_per_gen = wl.batch * wl.decode_steps
 
@@ -692,16 +752,23 @@ def main():
 
     # end to end: every input starts in pinned host memory, every output ends there
     if not args.no_extras:
-        job.make_host()
+        hjob = Job(wl, device, rows_per_chunk=args.rows_per_chunk, stage_shared=args.stage_shared,
+                   lazy_mask=args.lazy_mask, host_prefill=True)
+        hjob.make_host()
         for _ in range(2):
-            job.generation_host()
-        ms_e2e = timed(job.generation_host, args.steps, dist)
-        job.ctx.status()
+            hjob.generation_host()
+        ms_e2e = timed(hjob.generation_host, args.steps, dist)
+        hjob.ctx.status()
         line["e2e"] = {"value": job_value(tokens_per_gen, args.steps, world, ms_e2e), "unit": UNIT,
-                       "h2d_bytes_per_step": job.h2d_bytes(), "d2h_bytes_per_step": job.d2h_bytes(),
-                       "ms_per_step": ms_e2e / args.steps}
+                       "h2d_bytes_per_step": hjob.h2d_bytes(), "d2h_bytes_per_step": hjob.d2h_bytes(),
+                       "ms_per_step": ms_e2e / args.steps,
+                       "api": "st3_prefill_select_host + st3_decode_step_host + st3_host_sync: pinned host buffers, "
+                              "the library's two copy streams run ahead of and behind the kernels"}
+        hjob.ctx.close()
+        del hjob
+        torch.cuda.empty_cache()
 
-    if rank == 0 and world == 1 and not args.no_extras:
+    if rank == 0 and world == 1 and not args.no_extras and not args.e2e_only:
         # the same kernels with trimming disabled (full KV cache)
         full = Job(wl, device, disable_trim=True, rows_per_chunk=args.rows_per_chunk)
         for _ in range(3):
@@ -721,6 +788,13 @@ def main():
         line["static_rank"] = {"value": tokens_per_gen * args.steps / (ms_stat * 1e-3), "unit": UNIT}
         stat.ctx.close()
         del stat
+        # QK heredity (Eq. 6): lazy layers move their V rows only.  Stage-shared kept sets with no lazy layer,
+        # with the paper's pattern inside the last full stage, and with lazy layers inside the first stage.
+        if wl.name == "llava15_7b":
+            line["qk_heredity"] = [qk_heredity_line(wl, device, args, name, mask) for name, mask in (
+                ("stage_shared, no lazy layer", 0),
+                ("layers 29-30 inherit layer 28", (1 << 29) | (1 << 30)),
+                ("layers 4-6 inherit layer 3, layers 8-9 inherit layer 7", sum(1 << l for l in (4, 5, 6, 8, 9))))]
         # prefill-select alone, the one-call-per-layer pattern, and K/V held along a generation
         ms_pre = timed(job.prefill_only, args.steps, False)
         line["prefill_select_ms"] = ms_pre / args.steps

@@ -88,6 +88,8 @@ typedef struct {
   int32_t static_rank;       /* 1: Algorithm 3 as printed, see below; 0: re-rank at every step   */
   int32_t stage_shared;      /* 1: the layers between two pruning layers keep the pruning layer's */
                              /*    choice (Sec. 3.2, strided pruning); 0: every layer chooses     */
+  int32_t host_prefill;      /* 1: the workspace holds two per-layer staging areas for the prompt's */
+                             /*    K/V, which st3_prefill_select_host needs; 0: no such areas      */
   uint64_t lazy_mask;        /* bit l set: layer l is lazy (QK heredity, Eq. 6, Algorithm 2)      */
   double tau;                /* Eq. 8: beta = cos(t*pi/(2 tau)) for t < tau, else 0             */
   double sigma;              /* only ST3_ANNEAL_EXP: beta = exp(-t/sigma)                       */
@@ -124,7 +126,8 @@ int32_t st3_schedule_count(const st3_config* cfg, int32_t layer, int32_t step);
 st3_status st3_workspace_size(const st3_config* cfg, size_t* bytes);
 
 /* Builds a context over a caller-owned device workspace (256-byte aligned, `bytes` long, on the
- * current device).  Host-side set-up plus one cudaMemsetAsync of the bookkeeping area on the
+ * current device).  Host-side set-up (it also creates two CUDA streams and a few events for the
+ * host-buffer calls; no device memory) plus one cudaMemsetAsync of the bookkeeping area on the
  * default stream, which is synchronised before returning.  *out is NULL on failure. */
 st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, st3_ctx** out);
 
@@ -175,14 +178,30 @@ st3_status st3_decode_step(st3_ctx* ctx, int32_t step, int32_t layer_begin, int3
  * a call then starts only after all earlier work of the stream has finished. */
 st3_status st3_set_overlap(st3_ctx* ctx, int32_t on);
 
-/* Same step with HOST buffers (pinned memory recommended): the library copies q/k_new/v_new to
- * staging areas inside its workspace, runs the step and copies `out` back, all on the stream.
- * The host buffers must stay untouched until the stream has passed the call.  When the three inputs
- * lie back to back in host memory (k_new_host = q_host + size, v_new_host = k_new_host + size) and the
- * call covers all layers, they travel as one copy. */
+/* Same step with HOST buffers (pinned memory, else the copies do not overlap anything): the library copies
+ * q/k_new/v_new to one of two staging areas inside its workspace, runs the step on `cuda_stream` and copies
+ * `out` back.  The copies travel on two streams of the library's own, so that the inputs of step t+1 and the
+ * output of step t-1 move while the kernels of step t run.  Consequences for the caller:
+ *   - the input buffers must hold their final contents when the call is made (they are read without waiting
+ *     for earlier work of `cuda_stream`) and must stay untouched until the step's kernels have run;
+ *   - out_host is complete once `cuda_stream` has passed a later st3_host_sync (or after st3_get_status, which
+ *     waits for everything).
+ * When the three inputs lie back to back in host memory (k_new_host = q_host + size, v_new_host = k_new_host
+ * + size), they travel as one copy. */
 st3_status st3_decode_step_host(st3_ctx* ctx, int32_t step, int32_t layer_begin, int32_t layer_count,
                                 const void* q_host, const void* k_new_host, const void* v_new_host,
                                 void* out_host, void* cuda_stream);
+
+/* st3_prefill_select with HOST buffers (pinned), same shapes: the prompt's K/V rows travel layer by layer
+ * through two staging areas (st3_config.host_prefill = 1, else ST3_ERR_BAD_STATE), so that layer l is ingested,
+ * attended and trimmed while layer l+1 is on the bus.  Same rules for the buffers as st3_decode_step_host.
+ * Not available with lazy layers (a lazy layer and its source must share a call): ST3_ERR_UNSUPPORTED. */
+st3_status st3_prefill_select_host(st3_ctx* ctx, int32_t layer_begin, int32_t layer_count, const void* q_last_host,
+                                   const void* k_host, const void* v_host, const int32_t* text_len,
+                                   void* out_host, void* cuda_stream);
+
+/* Makes `cuda_stream` wait for every copy back to host memory that the two calls above have started. */
+st3_status st3_host_sync(st3_ctx* ctx, void* cuda_stream);
 
 /* Observability: copies layer `layer`'s kept original visual indices (ids dev [B][num_visual],
  * first count[b] entries valid, cache order), counts (count dev [B]) and, if mass != NULL, the
@@ -197,7 +216,7 @@ st3_status st3_get_kept(st3_ctx* ctx, int32_t layer, int32_t* ids, int32_t* coun
 st3_status st3_get_rows(st3_ctx* ctx, int32_t layer, int32_t b, int32_t h, void* k_vis, void* v_vis,
                         void* k_txt, void* v_txt, void* cuda_stream);
 
-/* Synchronises the stream last used by this context and returns the device status word through
+/* Synchronises the stream last used by this context (and the library's copy streams) and returns the device status word through
  * *word (host).  Returns ST3_ERR_DEVICE_CHECK if it is non-zero; the word is sticky and the results of
  * a context that has reported one are undefined from then on: destroy it and create a new one. */
 st3_status st3_get_status(st3_ctx* ctx, int32_t* word);
@@ -234,6 +253,23 @@ st3_status st3_prefill_attend(const void* q, const void* k, const void* v, void*
                               float* scores, int* dev_status, int32_t num_inst, int32_t num_heads,
                               int32_t seq_len, int32_t head_dim, int32_t dtype, int32_t sys_len,
                               int32_t num_visual, void* cuda_stream);
+
+/* The same for a layer that runs on the visual tokens an earlier layer kept (Algorithm 1: the sequence that
+ * enters layer l is [S | kept V | I]; Eq. 3 prunes layer l+1 by layer l's alpha).  num_visual is the number of
+ * kept tokens in the prompt given here, and
+ *   ids               dev [num_inst / num_heads][num_visual] int32: original index (< num_visual_total) of the
+ *                     token at each visual position, e.g. what st3_get_kept returned for this layer
+ *   scores            dev [num_inst / num_heads][num_visual_total] fp32, indexed by ORIGINAL visual index: the
+ *                     head-summed probability of the tokens held, -1 for every token not held (below any
+ *                     probability, so st3_prefill_select_scored of the next layer never keeps one of them while
+ *                     its count does not exceed num_visual)
+ * An id outside [0, num_visual_total) sets ST3_DEV_RANGE in *dev_status and is skipped.  With num_visual = 0
+ * the scores are all -1. */
+st3_status st3_prefill_attend_kept(const void* q, const void* k, const void* v, void* out, float* head_probs,
+                                   float* scores, int* dev_status, int32_t num_inst, int32_t num_heads,
+                                   int32_t seq_len, int32_t head_dim, int32_t dtype, int32_t sys_len,
+                                   int32_t num_visual, const int32_t* ids, int32_t num_visual_total,
+                                   void* cuda_stream);
 
 /* Attention of one query per head over dense K/V with NO workspace and no allocation of any kind
  * (the paper has no counterpart; this exists for callers that may not allocate device memory:

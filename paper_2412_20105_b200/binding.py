@@ -21,9 +21,9 @@ DEV_COUNT_MISMATCH, DEV_NONFINITE, DEV_COPY_TIMEOUT, DEV_RANGE = 1, 2, 4, 8
 
 EXPORTS = ["st3_schedule_count", "st3_workspace_size", "st3_create", "st3_prefill_select",
            "st3_prefill_select_scored", "st3_decode_step",
-           "st3_decode_step_host", "st3_get_kept", "st3_get_rows", "st3_get_status", "st3_rows_held",
+           "st3_decode_step_host", "st3_prefill_select_host", "st3_host_sync", "st3_get_kept", "st3_get_rows", "st3_get_status", "st3_rows_held",
            "st3_set_overlap", "st3_profile_enable", "st3_profile_read", "st3_launch_count", "st3_status_string", "st3_destroy",
-           "st3_attend_noalloc", "st3_prefill_attend"]
+           "st3_attend_noalloc", "st3_prefill_attend", "st3_prefill_attend_kept"]
 
 
 class Config(C.Structure):
@@ -31,7 +31,7 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "num_layers", "num_heads", "head_dim", "dtype", "batch", "sys_len", "num_visual", "max_text_len",
         "max_decode_steps", "first_prune_layer", "stride", "first_ratio_bp", "step_ratio_bp", "anneal",
-        "disable_trim", "rows_per_chunk", "static_rank", "stage_shared")] + [("lazy_mask", C.c_uint64), ("tau", C.c_double), ("sigma", C.c_double)]
+        "disable_trim", "rows_per_chunk", "static_rank", "stage_shared", "host_prefill")] + [("lazy_mask", C.c_uint64), ("tau", C.c_double), ("sigma", C.c_double)]
 
 
 class St3Error(RuntimeError):
@@ -63,6 +63,8 @@ def load():
     lib.st3_prefill_select_scored.argtypes = [vp, i32, i32, vp, vp, vp, C.POINTER(i32), vp, vp, vp]
     lib.st3_decode_step.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.st3_decode_step_host.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.st3_prefill_select_host.argtypes = [vp, i32, i32, vp, vp, vp, C.POINTER(i32), vp, vp]
+    lib.st3_host_sync.argtypes = [vp, vp]
     lib.st3_get_kept.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.st3_get_rows.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.st3_get_status.argtypes = [vp, C.POINTER(i32)]
@@ -78,6 +80,7 @@ def load():
     lib.st3_destroy.argtypes = [vp]
     lib.st3_attend_noalloc.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.st3_prefill_attend.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp]
+    lib.st3_prefill_attend_kept.argtypes = [vp, vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, i32, vp, i32, vp]
     for name in EXPORTS:
         if name not in ("st3_schedule_count", "st3_launch_count", "st3_status_string"):
             getattr(lib, name).restype = C.c_int
@@ -92,11 +95,13 @@ def _check(code: int, where: str):
 
 def make_config(*, num_layers, num_heads, head_dim, dtype, batch, sys_len, num_visual, max_text_len,
                 max_decode_steps, stride, step_ratio_bp, tau, first_prune_layer=3, first_ratio_bp=5000,
-                anneal=ST3_ANNEAL_COSINE, disable_trim=0, rows_per_chunk=0, sigma=20.0, static_rank=0, stage_shared=0, lazy_mask=0) -> Config:
+                anneal=ST3_ANNEAL_COSINE, disable_trim=0, rows_per_chunk=0, sigma=20.0, static_rank=0, stage_shared=0, lazy_mask=0,
+                host_prefill=0) -> Config:
     dt = {"f32": ST3_F32, "bf16": ST3_BF16}.get(dtype, dtype)
     return Config(num_layers, num_heads, head_dim, dt, batch, sys_len, num_visual, max_text_len,
                   max_decode_steps, first_prune_layer, stride, first_ratio_bp, step_ratio_bp, anneal,
-                  int(disable_trim), rows_per_chunk, int(static_rank), int(stage_shared), int(lazy_mask), float(tau), float(sigma))
+                  int(disable_trim), rows_per_chunk, int(static_rank), int(stage_shared), int(host_prefill), int(lazy_mask),
+                  float(tau), float(sigma))
 
 
 def st3_schedule_count(cfg: Config, layer: int, step: int) -> int:
@@ -138,6 +143,17 @@ def st3_decode_step(ctx, step, layer_begin, layer_count, q, k_new, v_new, out, s
 def st3_decode_step_host(ctx, step, layer_begin, layer_count, q, k_new, v_new, out, stream=0):
     _check(load().st3_decode_step_host(ctx, step, layer_begin, layer_count, q, k_new, v_new, out, stream),
            "st3_decode_step_host")
+
+
+def st3_prefill_select_host(ctx, layer_begin, layer_count, q_last, k, v, text_len, out, stream=0):
+    """As st3_prefill_select with pinned HOST addresses; needs a config with host_prefill=1."""
+    arr = (C.c_int32 * len(text_len))(*[int(x) for x in text_len])
+    _check(load().st3_prefill_select_host(ctx, layer_begin, layer_count, q_last, k, v, arr, out, stream),
+           "st3_prefill_select_host")
+
+
+def st3_host_sync(ctx, stream=0):
+    _check(load().st3_host_sync(ctx, stream), "st3_host_sync")
 
 
 def st3_get_kept(ctx, layer, ids, count, mass=None, stream=0):
@@ -195,6 +211,15 @@ def st3_prefill_attend(q, k, v, out, head_probs, scores, dev_status, num_inst, n
     dt = {"f32": ST3_F32, "bf16": ST3_BF16}.get(dtype, dtype)
     _check(load().st3_prefill_attend(q, k, v, out, head_probs, scores, dev_status, num_inst, num_heads, seq_len,
                                      head_dim, dt, sys_len, num_visual, stream), "st3_prefill_attend")
+
+
+def st3_prefill_attend_kept(q, k, v, out, head_probs, scores, dev_status, num_inst, num_heads, seq_len, head_dim,
+                            dtype, sys_len, num_visual, ids, num_visual_total, stream=0):
+    """The same for a prompt that holds only the visual tokens `ids` names; scores come out by original index."""
+    dt = {"f32": ST3_F32, "bf16": ST3_BF16}.get(dtype, dtype)
+    _check(load().st3_prefill_attend_kept(q, k, v, out, head_probs, scores, dev_status, num_inst, num_heads, seq_len,
+                                          head_dim, dt, sys_len, num_visual, ids, num_visual_total, stream),
+           "st3_prefill_attend_kept")
 
 
 def st3_attend_noalloc(q, k, v, out, num_heads, num_rows, head_dim, dtype, stream=0):
@@ -257,6 +282,14 @@ class Context:
         """q/k_new/v_new/out are pinned HOST tensors."""
         st3_decode_step_host(self.handle, step, layer_begin, q.shape[0], q.data_ptr(), k_new.data_ptr(),
                              v_new.data_ptr(), out.data_ptr(), self._stream())
+
+    def prefill_select_host(self, q_last, k, v, text_len, out, layer_begin=0):
+        """q_last/k/v/out are pinned HOST tensors."""
+        st3_prefill_select_host(self.handle, layer_begin, q_last.shape[0], q_last.data_ptr(), k.data_ptr(),
+                                v.data_ptr(), text_len, out.data_ptr(), self._stream())
+
+    def host_sync(self):
+        st3_host_sync(self.handle, self._stream())
 
     def get_kept(self, layer, with_mass=True):
         t, c = self.torch, self.cfg

@@ -51,8 +51,15 @@ inline void make_fast_div(unsigned d, unsigned* mul, unsigned* shift) {
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
 struct Layout {
-  size_t elem, cache, part_ml, part_acc, part_ml_bytes, part_acc_bytes, logits, logits_bytes, head_stat, mass, ids, n_cur, flags, text_len, status, stage_q, stage_k, stage_v,
-      stage_o, total;
+  size_t elem, cache, part_ml, part_acc, part_ml_bytes, part_acc_bytes, logits, logits_bytes, head_stat, mass, ids, n_cur, flags, text_len, status,
+      io_bytes,       // one of q / k_new / v_new / out over all layers
+      stage_in,       // two slots of [q | k_new | v_new] for the host-buffer decode step
+      stage_o,        // two slots of out
+      stage_pq,       // q_last and out of the host-buffer prefill
+      stage_po,
+      prompt_bytes,   // K (or V) rows of one layer's prompt
+      stage_prompt,   // two slots of [K | V] of one layer (only with host_prefill)
+      total;
   long long lbh_stride;
   int cap_txt, chunk_rows, max_items;
 };
@@ -131,8 +138,14 @@ Layout make_layout(const st3_config* c) {
   L.flags = take(lb * sizeof(int));
   L.text_len = take((size_t)c->batch * sizeof(int));
   L.status = take(256);
-  const size_t io = lbh * c->head_dim * L.elem;
-  L.stage_q = take(io); L.stage_k = take(io); L.stage_v = take(io); L.stage_o = take(io);
+  L.io_bytes = align_up(lbh * c->head_dim * L.elem, 256);
+  L.stage_in = take(2 * 3 * L.io_bytes);
+  L.stage_o = take(2 * L.io_bytes);
+  L.stage_pq = take(L.io_bytes);
+  L.stage_po = take(L.io_bytes);
+  L.prompt_bytes = align_up((size_t)c->batch * c->num_heads * ((size_t)c->sys_len + c->num_visual + c->max_text_len) *
+                                c->head_dim * L.elem, 256);
+  L.stage_prompt = c->host_prefill ? take(2 * 2 * L.prompt_bytes) : off;
   L.total = off;
   return L;
 }
@@ -183,6 +196,12 @@ struct st3_ctx {
   bool serialize_next;         // the next attention launch must wait for every earlier launch
   bool overlap;                // st3_set_overlap: the attention launch may start before the launch ahead of it ends
   bool failed;                 // a launch failed half-way: host bookkeeping and device state may disagree
+  // host-buffer calls: copies to the device and back travel on two streams of the library's own
+  cudaStream_t s_h2d, s_d2h;
+  cudaEvent_t ev_in[2], ev_k[2], ev_out[2];   // per decode staging slot: inputs landed / kernels done / out copied back
+  cudaEvent_t ev_pin[2], ev_pk[2], ev_pq;     // per prompt staging slot: K/V landed / layer done; q_last staging free
+  bool rec_k[2], rec_out[2], rec_pk[2], rec_pq;
+  uint64_t hseq, pseq;                        // host-buffer decode steps / prompt layers so far (slot = low bit)
 };
 
 namespace {
@@ -230,7 +249,11 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = (!ctx->overlap || ctx->profiling || ingest || ctx->serialize_next) ? 0 : 1;
-    if (cudaLaunchKernelEx(&cfg, st3_attend_kernel<T, D>, p) != cudaSuccess) return ST3_ERR_CUDA;
+    bool fat = false;  // some item carries lazy layers (QK heredity): the instantiation that streams their values
+    for (int i = 0; i < p.layer_count; ++i) fat = fat || p.nfol[i] != 0;
+    if ((fat ? cudaLaunchKernelEx(&cfg, st3_attend_kernel<T, D, true>, p)
+             : cudaLaunchKernelEx(&cfg, st3_attend_kernel<T, D, false>, p)) != cudaSuccess)
+      return ST3_ERR_CUDA;
   }
   if (e1) cudaEventRecord(e1, st);
   {
@@ -255,7 +278,9 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
 
 template <typename T, int D>
 st3_status set_attrs_t(st3_ctx* ctx) {
-  if (cudaFuncSetAttribute(st3_attend_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (cudaFuncSetAttribute(st3_attend_kernel<T, D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           ctx->attend_smem) != cudaSuccess ||
+      cudaFuncSetAttribute(st3_attend_kernel<T, D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            ctx->attend_smem) != cudaSuccess)
     return ST3_ERR_CUDA;
   if (cudaFuncSetAttribute(st3_finish_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -341,13 +366,39 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
     make_fast_div((unsigned)(cv > 0 ? cv : 1), &p.cv_mul[i], &p.cv_shift[i]);
   }
   p.lstart[layer_count] = c.batch * (p.cvp[layer_count] + layer_count * p.ct);
+  // Working layers: every layer except the lazy ones that ride on the items of the layer they inherit from
+  // (their value rows follow the item through its ring slot, see st3_attend.cuh; a run of more than kMaxFollow
+  // lazy layers would start a new group that reads the keys again).
+  bool works[kMaxLayers];
+  for (int i = 0, head = -1; i < layer_count; ++i) {
+    const int s = p.lazy_src[i];
+    const bool rides = s >= 0 && head >= 0 && (head == s || p.lazy_src[head] == s) &&
+                       head + p.nfol[head] + 1 == i && p.nfol[head] < kMaxFollow &&
+                       p.ncur[i] == p.ncur[head] && p.nold[i] == p.nold[head];
+    works[i] = !rides;
+    if (rides) p.nfol[head]++;
+    else head = i;
+  }
+  // Order of the working layers inside the launch: those whose items are followed by lazy layers first.  Such an
+  // item keeps its ring slot for several uses in a row; at the end of a launch, where little other work is left
+  // to hide it, that chain would set the length of the tail.
+  p.nwork = 0;
+  p.wcvp[0] = 0;
+  for (int pass = 0; pass < 2; ++pass)
+    for (int i = 0; i < layer_count; ++i) {
+      if (!works[i] || (p.nfol[i] != 0) != (pass == 0)) continue;
+      p.wlayer[p.nwork] = (unsigned char)i;
+      p.wcvp[p.nwork + 1] = p.wcvp[p.nwork] + (p.cvp[i + 1] - p.cvp[i]);
+      p.nwork++;
+    }
   make_fast_div((unsigned)c.num_heads, &p.h_mul, &p.h_shift);
-  p.text_items = layer_count * c.batch * p.ct;
+  p.text_items = p.nwork * c.batch * p.ct;
   make_fast_div((unsigned)(c.batch * p.ct), &p.bct_mul, &p.bct_shift);
   make_fast_div((unsigned)p.ct, &p.ct_mul, &p.ct_shift);
   const long long total_items = (long long)c.batch * (p.cvp[layer_count] + (long long)layer_count * p.ct);
-  if (total_items > L.max_items || total_items * c.num_heads > 0x3fffffffLL) return ST3_ERR_CAPACITY;
-  p.total_work = (int)(total_items * c.num_heads);
+  const long long work_items = (long long)c.batch * (p.wcvp[p.nwork] + (long long)p.nwork * p.ct);
+  if (total_items > L.max_items || work_items * c.num_heads > 0x3fffffffLL) return ST3_ERR_CAPACITY;
+  p.total_work = (int)(work_items * c.num_heads);
   p.first_dynamic = ctx->num_sms * ctx->attend_ctas_per_sm * kSlots;
 
   StepParams psel;
@@ -436,6 +487,14 @@ st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, 
   ctx->failed = false;
   ctx->profiling = false;
   ctx->ev_used = 0;
+  ctx->s_h2d = ctx->s_d2h = nullptr;
+  ctx->ev_pq = nullptr;
+  for (int i = 0; i < 2; ++i) {
+    ctx->ev_in[i] = ctx->ev_k[i] = ctx->ev_out[i] = ctx->ev_pin[i] = ctx->ev_pk[i] = nullptr;
+    ctx->rec_k[i] = ctx->rec_out[i] = ctx->rec_pk[i] = false;
+  }
+  ctx->rec_pq = false;
+  ctx->hseq = ctx->pseq = 0;
   ctx->attend_smem = kSlots * (2 * tile_bytes(cfg) + kQBytes);
   int dev = 0, sms = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -452,11 +511,23 @@ st3_status st3_create(const st3_config* cfg, void* dev_workspace, size_t bytes, 
 #undef ST3_ATTR
   if (s == ST3_OK) {
     // bookkeeping area (scores, ids, counts, text lengths, status word) starts cleared
-    if (cudaMemsetAsync(ctx->ws + L.mass, 0, L.stage_q - L.mass, nullptr) != cudaSuccess ||
+    if (cudaMemsetAsync(ctx->ws + L.mass, 0, L.stage_in - L.mass, nullptr) != cudaSuccess ||
         cudaStreamSynchronize(nullptr) != cudaSuccess)
       s = ST3_ERR_CUDA;
   }
-  if (s != ST3_OK) { delete ctx; return s; }
+  if (s == ST3_OK) {
+    bool ok = cudaStreamCreateWithFlags(&ctx->s_h2d, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&ctx->s_d2h, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&ctx->ev_pq, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 2 && ok; ++i)
+      ok = cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ctx->ev_k[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ctx->ev_out[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ctx->ev_pin[i], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&ctx->ev_pk[i], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) s = ST3_ERR_CUDA;
+  }
+  if (s != ST3_OK) { st3_destroy(ctx); return s; }
   *out = ctx;
   return ST3_OK;
 }
@@ -527,28 +598,99 @@ st3_status st3_decode_step_host(st3_ctx* ctx, int32_t step, int32_t layer_begin,
                                 const void* q_host, const void* k_new_host, const void* v_new_host, void* out_host,
                                 void* cuda_stream) {
   if (!ctx || !q_host || !k_new_host || !v_new_host || !out_host) return ST3_ERR_INVALID_ARG;
+  if (ctx->failed) return ST3_ERR_BAD_STATE;
   const st3_config& c = ctx->cfg;
   if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c.num_layers) return ST3_ERR_INVALID_ARG;
   const Layout& L = ctx->lay;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   const size_t bytes = (size_t)layer_count * c.batch * c.num_heads * c.head_dim * L.elem;
-  unsigned char* dq = ctx->ws + L.stage_q; unsigned char* dk = ctx->ws + L.stage_k;
-  unsigned char* dv = ctx->ws + L.stage_v; unsigned char* dout = ctx->ws + L.stage_o;
+  const int slot = (int)(ctx->hseq & 1);
+  unsigned char* dq = ctx->ws + L.stage_in + (size_t)slot * 3 * L.io_bytes;
+  unsigned char* dk = dq + bytes;
+  unsigned char* dv = dk + bytes;
+  unsigned char* dout = ctx->ws + L.stage_o + (size_t)slot * L.io_bytes;
   const unsigned char* hq = static_cast<const unsigned char*>(q_host);
   const unsigned char* hk = static_cast<const unsigned char*>(k_new_host);
   const unsigned char* hv = static_cast<const unsigned char*>(v_new_host);
-  if (hk == hq + bytes && hv == hk + bytes && dk == dq + bytes && dv == dk + bytes) {
-    // q, k_new, v_new packed back to back by the caller: one copy instead of three (two copy launches
-    // less on a step that lasts tens of microseconds)
-    if (cudaMemcpyAsync(dq, hq, 3 * bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return ST3_ERR_CUDA;
-  } else if (cudaMemcpyAsync(dq, hq, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-             cudaMemcpyAsync(dk, hk, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-             cudaMemcpyAsync(dv, hv, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+  // inputs: on the copy-in stream, once the kernels that last read this staging slot (two steps ago) are done
+  if (ctx->rec_k[slot] && cudaStreamWaitEvent(ctx->s_h2d, ctx->ev_k[slot], 0) != cudaSuccess) return ST3_ERR_CUDA;
+  if (hk == hq + bytes && hv == hk + bytes) {
+    // q, k_new, v_new packed back to back by the caller: one copy instead of three
+    if (cudaMemcpyAsync(dq, hq, 3 * bytes, cudaMemcpyHostToDevice, ctx->s_h2d) != cudaSuccess) return ST3_ERR_CUDA;
+  } else if (cudaMemcpyAsync(dq, hq, bytes, cudaMemcpyHostToDevice, ctx->s_h2d) != cudaSuccess ||
+             cudaMemcpyAsync(dk, hk, bytes, cudaMemcpyHostToDevice, ctx->s_h2d) != cudaSuccess ||
+             cudaMemcpyAsync(dv, hv, bytes, cudaMemcpyHostToDevice, ctx->s_h2d) != cudaSuccess) {
     return ST3_ERR_CUDA;
   }
+  if (cudaEventRecord(ctx->ev_in[slot], ctx->s_h2d) != cudaSuccess ||
+      cudaStreamWaitEvent(st, ctx->ev_in[slot], 0) != cudaSuccess)
+    return ST3_ERR_CUDA;
+  // the slot's output staging must have been copied back (two steps ago) before the kernels write it again
+  if (ctx->rec_out[slot] && cudaStreamWaitEvent(st, ctx->ev_out[slot], 0) != cudaSuccess) return ST3_ERR_CUDA;
   const st3_status s = st3_decode_step(ctx, step, layer_begin, layer_count, dq, dk, dv, dout, cuda_stream);
   if (s != ST3_OK) return s;
-  if (cudaMemcpyAsync(out_host, dout, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ST3_ERR_CUDA;
+  if (cudaEventRecord(ctx->ev_k[slot], st) != cudaSuccess) return ST3_ERR_CUDA;
+  ctx->rec_k[slot] = true;
+  // output: on the copy-out stream, behind the kernels
+  if (cudaStreamWaitEvent(ctx->s_d2h, ctx->ev_k[slot], 0) != cudaSuccess ||
+      cudaMemcpyAsync(out_host, dout, bytes, cudaMemcpyDeviceToHost, ctx->s_d2h) != cudaSuccess ||
+      cudaEventRecord(ctx->ev_out[slot], ctx->s_d2h) != cudaSuccess)
+    return ST3_ERR_CUDA;
+  ctx->rec_out[slot] = true;
+  ctx->hseq++;
+  return ST3_OK;
+}
+
+st3_status st3_prefill_select_host(st3_ctx* ctx, int32_t layer_begin, int32_t layer_count, const void* q_last_host,
+                                   const void* k_host, const void* v_host, const int32_t* text_len, void* out_host,
+                                   void* cuda_stream) {
+  if (!ctx || !q_last_host || !k_host || !v_host || !out_host || !text_len) return ST3_ERR_INVALID_ARG;
+  if (ctx->failed || !ctx->cfg.host_prefill) return ST3_ERR_BAD_STATE;
+  const st3_config& c = ctx->cfg;
+  if (layer_begin < 0 || layer_count < 1 || layer_begin + layer_count > c.num_layers) return ST3_ERR_INVALID_ARG;
+  if (c.lazy_mask) return ST3_ERR_UNSUPPORTED;
+  const Layout& L = ctx->lay;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  const size_t lq = (size_t)c.batch * c.num_heads * c.head_dim * L.elem;  // one layer of q_last / out
+  const size_t lp = (size_t)c.batch * c.num_heads * ((size_t)c.sys_len + c.num_visual + c.max_text_len) * c.head_dim * L.elem;
+  unsigned char* dq = ctx->ws + L.stage_pq;
+  unsigned char* dout = ctx->ws + L.stage_po;
+  // q_last of every layer in one copy, once the kernels of an earlier call are done with the staging area
+  if (ctx->rec_pq && cudaStreamWaitEvent(ctx->s_h2d, ctx->ev_pq, 0) != cudaSuccess) return ST3_ERR_CUDA;
+  if (cudaMemcpyAsync(dq, q_last_host, lq * layer_count, cudaMemcpyHostToDevice, ctx->s_h2d) != cudaSuccess)
+    return ST3_ERR_CUDA;
+  for (int i = 0; i < layer_count; ++i) {
+    const int slot = (int)(ctx->pseq & 1);
+    unsigned char* dk = ctx->ws + L.stage_prompt + (size_t)slot * 2 * L.prompt_bytes;
+    unsigned char* dv = dk + L.prompt_bytes;
+    // layer i's rows move while the layer before it is ingested, attended and trimmed
+    if (ctx->rec_pk[slot] && cudaStreamWaitEvent(ctx->s_h2d, ctx->ev_pk[slot], 0) != cudaSuccess) return ST3_ERR_CUDA;
+    if (cudaMemcpyAsync(dk, static_cast<const unsigned char*>(k_host) + (size_t)i * lp, lp, cudaMemcpyHostToDevice,
+                        ctx->s_h2d) != cudaSuccess ||
+        cudaMemcpyAsync(dv, static_cast<const unsigned char*>(v_host) + (size_t)i * lp, lp, cudaMemcpyHostToDevice,
+                        ctx->s_h2d) != cudaSuccess ||
+        cudaEventRecord(ctx->ev_pin[slot], ctx->s_h2d) != cudaSuccess ||
+        cudaStreamWaitEvent(st, ctx->ev_pin[slot], 0) != cudaSuccess)
+      return ST3_ERR_CUDA;
+    const st3_status s = prefill_common(ctx, layer_begin + i, 1, dq + (size_t)i * lq, dk, dv, text_len, nullptr,
+                                        dout + (size_t)i * lq, cuda_stream);
+    if (s != ST3_OK) return s;
+    if (cudaEventRecord(ctx->ev_pk[slot], st) != cudaSuccess) return ST3_ERR_CUDA;
+    ctx->rec_pk[slot] = true;
+    ctx->pseq++;
+  }
+  if (cudaEventRecord(ctx->ev_pq, st) != cudaSuccess) return ST3_ERR_CUDA;
+  ctx->rec_pq = true;
+  // the outputs of all layers in one copy, behind the last layer's kernels
+  if (cudaMemcpyAsync(out_host, dout, lq * layer_count, cudaMemcpyDeviceToHost, st) != cudaSuccess) return ST3_ERR_CUDA;
+  return ST3_OK;
+}
+
+st3_status st3_host_sync(st3_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return ST3_ERR_INVALID_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  for (int i = 0; i < 2; ++i)
+    if (ctx->rec_out[i] && cudaStreamWaitEvent(st, ctx->ev_out[i], 0) != cudaSuccess) return ST3_ERR_CUDA;
   return ST3_OK;
 }
 
@@ -597,7 +739,9 @@ st3_status st3_get_rows(st3_ctx* ctx, int32_t layer, int32_t b, int32_t h, void*
 
 st3_status st3_get_status(st3_ctx* ctx, int32_t* word) {
   if (!ctx || !word) return ST3_ERR_INVALID_ARG;
-  if (cudaStreamSynchronize(ctx->last_stream) != cudaSuccess) return ST3_ERR_CUDA;
+  if (cudaStreamSynchronize(ctx->last_stream) != cudaSuccess || cudaStreamSynchronize(ctx->s_h2d) != cudaSuccess ||
+      cudaStreamSynchronize(ctx->s_d2h) != cudaSuccess)
+    return ST3_ERR_CUDA;
   int w = 0;
   if (cudaMemcpy(&w, ctx->ws + ctx->lay.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
     return ST3_ERR_CUDA;
@@ -673,6 +817,12 @@ const char* st3_status_string(st3_status s) {
 st3_status st3_destroy(st3_ctx* ctx) {
   if (!ctx) return ST3_ERR_INVALID_ARG;
   for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+  for (int i = 0; i < 2; ++i)
+    for (cudaEvent_t e : {ctx->ev_in[i], ctx->ev_k[i], ctx->ev_out[i], ctx->ev_pin[i], ctx->ev_pk[i]})
+      if (e) cudaEventDestroy(e);
+  if (ctx->ev_pq) cudaEventDestroy(ctx->ev_pq);
+  if (ctx->s_h2d) cudaStreamDestroy(ctx->s_h2d);
+  if (ctx->s_d2h) cudaStreamDestroy(ctx->s_d2h);
   delete ctx;
   return ST3_OK;
 }

@@ -19,6 +19,7 @@ constexpr int kMaxLayers = 64;
 constexpr int kMaxHeads = 128;
 constexpr int kMaxVisual = 8192;
 constexpr long long kWaitCycles = 4000000000LL;  // ~2 s: bound on any wait for an async copy
+constexpr int kMaxFollow = 62;  // lazy layers whose values can follow one work item of the layer they inherit from
 
 struct StepParams {
   const void* q;
@@ -68,6 +69,13 @@ struct StepParams {
   int src_layer[kMaxLayers];  // the layer whose scores decide this layer's evictions (itself unless stage-shared)
   int src_copy[kMaxLayers];   // which copy of the logits holds that layer's logits
   int lazy_src[kMaxLayers];   // relative index of the layer whose q and K a lazy layer inherits (-1: its own)
+  // QK heredity (Eq. 6) without re-reading keys: the lazy layers right above a layer ride on that layer's work
+  // items (its probabilities are applied to their value rows as well); they get no items of their own.  The
+  // attention launch numbers its work over the remaining ("working") layers only.
+  int nwork;                          // working layers of this call
+  int wcvp[kMaxLayers + 1];           // prefix sum of their visual chunks
+  unsigned char wlayer[kMaxLayers];   // relative layer index of the w-th working layer
+  unsigned char nfol[kMaxLayers];     // lazy layers riding on this (working) layer's items
 };
 
 // ------------------------------------------------------------------------------------------

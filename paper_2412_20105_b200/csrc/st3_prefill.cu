@@ -466,6 +466,28 @@ __global__ void st3_prefill_scores_kernel(const float* __restrict__ head_probs, 
   scores[(size_t)b * num_visual + i] = s;
 }
 
+// The same sum for a layer that ran on the visual tokens an earlier layer kept: position i of the layer's visual
+// span is original token ids[b][i], and the scores go out indexed by original token (tokens not held: -1).
+__global__ void st3_prefill_fill_kernel(float* __restrict__ scores, long long n, float value) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) scores[i] = value;
+}
+__global__ void st3_prefill_scores_by_id_kernel(const float* __restrict__ head_probs, const int* __restrict__ ids,
+                                                float* __restrict__ scores, int* status, int num_heads, int num_visual,
+                                                int num_visual_total) {
+  const int b = blockIdx.y;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= num_visual) return;
+  const int id = ids[(size_t)b * num_visual + i];
+  if ((unsigned)id >= (unsigned)num_visual_total) {  // reported, not used
+    if (status) atomicOr(status, ST3_DEV_RANGE);
+    return;
+  }
+  float s = 0.f;
+  for (int h = 0; h < num_heads; ++h) s += head_probs[((size_t)b * num_heads + h) * num_visual + i];
+  scores[(size_t)b * num_visual_total + id] = s;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -484,10 +506,11 @@ bool make_map(EncodeTiledFn fn, CUtensorMap* map, const void* base, size_t num_i
 
 }  // namespace
 
-extern "C" st3_status st3_prefill_attend(const void* q, const void* k, const void* v, void* out, float* head_probs,
-                                         float* scores, int* dev_status, int32_t num_inst, int32_t num_heads,
-                                         int32_t seq_len, int32_t head_dim, int32_t dtype, int32_t sys_len,
-                                         int32_t num_visual, void* cuda_stream) {
+static st3_status prefill_attend_impl(const void* q, const void* k, const void* v, void* out, float* head_probs,
+                                      float* scores, int* dev_status, int32_t num_inst, int32_t num_heads,
+                                      int32_t seq_len, int32_t head_dim, int32_t dtype, int32_t sys_len,
+                                      int32_t num_visual, const int32_t* ids, int32_t num_visual_total,
+                                      void* cuda_stream) {
   auto aligned = [](const void* ptr) { return ptr && (reinterpret_cast<uintptr_t>(ptr) & 15u) == 0; };
   if (!aligned(q) || !aligned(k) || !aligned(v) || !aligned(out)) return ST3_ERR_INVALID_ARG;
   if (num_inst < 1 || num_heads < 1 || num_inst % num_heads || seq_len < 1) return ST3_ERR_INVALID_ARG;
@@ -521,9 +544,38 @@ extern "C" st3_status st3_prefill_attend(const void* q, const void* k, const voi
   p.T = seq_len; p.sys_len = sys_len; p.num_visual = num_visual;
   const dim3 grid((unsigned)((seq_len + kTile - 1) / kTile), (unsigned)num_inst);
   st3_prefill_attend_kernel<<<grid, kPfThreads, smem, st>>>(mq, mk, mv, p);
-  if (num_visual > 0) {
-    const dim3 g2((unsigned)((num_visual + 255) / 256), (unsigned)(num_inst / num_heads));
+  const int num_seq = num_inst / num_heads;
+  if (ids) {
+    const long long n = (long long)num_seq * num_visual_total;
+    st3_prefill_fill_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(scores, n, -1.f);
+    if (num_visual > 0) {
+      const dim3 g2((unsigned)((num_visual + 255) / 256), (unsigned)num_seq);
+      st3_prefill_scores_by_id_kernel<<<g2, 256, 0, st>>>(head_probs, ids, scores, dev_status, num_heads, num_visual,
+                                                          num_visual_total);
+    }
+  } else if (num_visual > 0) {
+    const dim3 g2((unsigned)((num_visual + 255) / 256), (unsigned)num_seq);
     st3_prefill_scores_kernel<<<g2, 256, 0, st>>>(head_probs, scores, num_heads, num_visual);
   }
   return cudaGetLastError() == cudaSuccess ? ST3_OK : ST3_ERR_CUDA;
+}
+
+extern "C" st3_status st3_prefill_attend(const void* q, const void* k, const void* v, void* out, float* head_probs,
+                                         float* scores, int* dev_status, int32_t num_inst, int32_t num_heads,
+                                         int32_t seq_len, int32_t head_dim, int32_t dtype, int32_t sys_len,
+                                         int32_t num_visual, void* cuda_stream) {
+  return prefill_attend_impl(q, k, v, out, head_probs, scores, dev_status, num_inst, num_heads, seq_len, head_dim,
+                             dtype, sys_len, num_visual, nullptr, 0, cuda_stream);
+}
+
+extern "C" st3_status st3_prefill_attend_kept(const void* q, const void* k, const void* v, void* out,
+                                              float* head_probs, float* scores, int* dev_status, int32_t num_inst,
+                                              int32_t num_heads, int32_t seq_len, int32_t head_dim, int32_t dtype,
+                                              int32_t sys_len, int32_t num_visual, const int32_t* ids,
+                                              int32_t num_visual_total, void* cuda_stream) {
+  if (!ids || (reinterpret_cast<uintptr_t>(ids) & 3u) || !scores || num_visual_total < num_visual ||
+      num_visual_total < 1)
+    return ST3_ERR_INVALID_ARG;
+  return prefill_attend_impl(q, k, v, out, head_probs, scores, dev_status, num_inst, num_heads, seq_len, head_dim,
+                             dtype, sys_len, num_visual, ids, num_visual_total, cuda_stream);
 }

@@ -287,8 +287,10 @@ class GpuRun:
         assert torch.equal(kt[:nk].cpu(), Kt[0, 0, h, :nk])
 
 
-def run_and_check(wl: Workload, steps, check_steps=None, units=None, layers_per_call=None, rows_checks=2, **cfg):
-    """Prefill + decode `steps` steps; check every (b, l) unit (or the sampled `units`) at `check_steps`."""
+def run_and_check(wl: Workload, steps, check_steps=None, units=None, layers_per_call=None, rows_checks=2,
+                  rows_units=None, **cfg):
+    """Prefill + decode `steps` steps; check every (b, l) unit (or the sampled `units`) at `check_steps`.
+    Cache rows are compared for the first `rows_checks` units, or for `rows_units` if given."""
     run = GpuRun(wl, **cfg)
     try:
         all_units = [(b, l) for l in range(wl.num_layers) for b in range(wl.batch)]
@@ -305,7 +307,7 @@ def run_and_check(wl: Workload, steps, check_steps=None, units=None, layers_per_
             if t in check_steps:
                 for b, l in units:
                     run.check_decode_unit(b, l, t, before[l])
-                for b, l in units[:rows_checks]:
+                for b, l in (units[:rows_checks] if rows_units is None else rows_units):
                     run.check_rows_unit(b, l, (t * 7) % wl.num_heads, t)
         assert run.ctx.status() == 0
         return run.stats

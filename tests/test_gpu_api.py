@@ -53,6 +53,68 @@ def test_host_buffer_step_equals_device_step(packed):
         a.close(); b.close()
 
 
+@pytest.mark.parametrize("overlap", [False, True])
+def test_host_buffer_generation_runs_ahead_of_the_gpu(overlap):
+    """Prefill and every decode step through the host-buffer calls, enqueued back to back with no synchronisation
+    in between (the library's copy streams run ahead of and behind the kernels), against the same generation
+    with device buffers: outputs bit-identical, same kept ids.  st3_host_sync + a wait on the caller's stream
+    is all that makes the host outputs readable."""
+    wl = _small()
+    steps = 9
+    a, b = GpuRun(wl), GpuRun(wl, overlap=overlap, host_prefill=1)
+    try:
+        g = b.g
+        q0 = g.queries([0])[0]
+        K, V = g.prompt_kv(range(wl.num_layers))
+        hq0, hK, hV = q0.pin_memory(), K.pin_memory(), V.pin_memory()
+        hout0 = torch.empty_like(hq0).pin_memory()
+        qs = g.queries(list(range(1, steps + 1)))
+        kn, vn = g.new_kv(list(range(1, steps + 1)))
+        hqkv = torch.stack([qs, kn, vn], dim=1).contiguous().pin_memory()        # [step][q | k | v]
+        hout = torch.zeros_like(qs).pin_memory()
+        b.ctx.prefill_select_host(hq0, hK, hV, g.text_len.tolist(), hout0)
+        for t in range(1, steps + 1):
+            b.ctx.decode_step_host(t, hqkv[t - 1, 0], hqkv[t - 1, 1], hqkv[t - 1, 2], hout[t - 1])
+        b.ctx.host_sync()
+        torch.cuda.current_stream().synchronize()
+        a.prefill()
+        assert torch.equal(hout0, a.out.cpu())
+        for t in range(1, steps + 1):
+            a.decode(t)
+            assert torch.equal(hout[t - 1], a.out.cpu()), t
+        for l in range(wl.num_layers):
+            ia, ca, _ = a.kept(l)
+            ib, cb, _ = b.kept(l)
+            assert np.array_equal(ca, cb)
+            for s in range(wl.batch):
+                assert np.array_equal(ia[s, :ca[s]], ib[s, :cb[s]])
+        assert a.ctx.status() == 0 and b.ctx.status() == 0
+        # a second generation on the same context reuses the staging areas behind the first one's work
+        b.ctx.prefill_select_host(hq0, hK, hV, g.text_len.tolist(), hout0)
+        b.ctx.decode_step_host(1, hqkv[0, 0], hqkv[0, 1], hqkv[0, 2], hout[0])
+        b.ctx.host_sync()
+        torch.cuda.current_stream().synchronize()
+        a.prefill(); a.decode(1)
+        assert torch.equal(hout[0], a.out.cpu()) and b.ctx.status() == 0
+    finally:
+        a.close(); b.close()
+
+
+def test_host_buffer_prefill_needs_its_staging_areas():
+    wl = _small()
+    run = GpuRun(wl)                       # host_prefill = 0
+    try:
+        g = run.g
+        q0 = g.queries([0])[0].pin_memory()
+        K, V = g.prompt_kv(range(wl.num_layers))
+        with pytest.raises(B.St3Error) as e:
+            run.ctx.prefill_select_host(q0, K.pin_memory(), V.pin_memory(), g.text_len.tolist(),
+                                        torch.empty_like(q0).pin_memory())
+        assert e.value.code == 3
+    finally:
+        run.close()
+
+
 def test_call_order_and_capacity_errors():
     wl = _small()
     run = GpuRun(wl)

@@ -189,6 +189,21 @@ def test_qk_heredity_lazy_layers():
     assert stats["units"] == 11 * 9 * 2
 
 
+@pytest.mark.parametrize("dtype,head_dim,overlap", [("bf16", 128, True), ("f32", 64, False), ("f32", 128, True),
+                                                    ("bf16", 64, False)])
+def test_qk_heredity_runs_of_lazy_layers(dtype, head_dim, overlap):
+    """Runs of lazy layers of odd and even length (their value rows follow their source's work item through its
+    ring slot two layers at a time), below the first pruning layer and inside a pruning stage; every kernel
+    instantiation; cache rows of lazy layers (values appended, no keys stored) compared bit for bit."""
+    wl = get_workload("tiny").scaled(dtype=dtype, head_dim=head_dim, num_heads=3, num_layers=12, batch=2, sys_len=3,
+                                     num_visual=150, text_len_min=1, text_len_max=70, decode_steps=8,
+                                     first_prune_layer=7, stride=5, step_ratio_bp=1000, tau=9.0, num_planted=7)
+    lazy = sum(1 << l for l in (1, 2, 3, 4, 5, 8, 9, 10, 11))     # 0 -> 1..5, 6 on its own, 7 -> 8..11
+    stats = run_and_check(wl, 8, stage_shared=1, lazy_mask=lazy, overlap=overlap,
+                          rows_units=[(0, 0), (1, 3), (0, 4), (1, 5), (0, 7), (1, 9), (0, 11)])
+    assert stats["units"] == 9 * 12 * 2
+
+
 def test_qk_heredity_configuration_errors():
     from paper_2412_20105_b200 import binding as B
     wl = get_workload("tiny").scaled(num_layers=9, first_prune_layer=2, stride=3, step_ratio_bp=1500)

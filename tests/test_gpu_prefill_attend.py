@@ -116,6 +116,81 @@ def test_scores_feed_the_scored_prefill():
         ctx.close()
 
 
+def test_pruning_layers_chained_over_kept_tokens():
+    """Algorithm 1 over three pruning layers back to back: the causal attention of layer l runs on the tokens
+    layer l kept ([S | kept V | I], in sequence order), its last row gives alpha^l by ORIGINAL visual index
+    (st3_prefill_attend_kept), and that prunes layer l+1 before it attends (st3_prefill_select_scored, Eq. 3).
+    The oracle walks the same chain with causal_attention and prefill_select_scored; every kept set is judged
+    with the near-tie rule on the oracle's scores and is nested in the previous layer's."""
+    from helpers import check_kept
+    build()
+    L, H, sys_len, nv, text = 3, 3, 5, 150, 21
+    T = sys_len + nv + text
+    g = torch.Generator().manual_seed(11)
+    mk = lambda *shape: torch.randn(*shape, generator=g).to(torch.bfloat16).cuda()
+    Q, K, V = mk(L, H, T, 128), mk(L, H, T, 128), mk(L, H, T, 128)       # the full prompt of every layer
+    Qp, Kp, Vp = mk(H, T, 128), mk(H, T, 128), mk(H, T, 128)             # the layer ahead of the first pruning layer
+    # keys of a few visual tokens pulled toward the last query so that the scores have structure
+    for t in (Kp, K[0], K[1], K[2]):
+        t[:, sys_len + 7:sys_len + nv:9] += 0.25 * (Qp[:, -1:] if t is Kp else Q[0, :, -1:])
+    cfg = B.make_config(num_layers=L, num_heads=H, head_dim=128, dtype="bf16", batch=1, sys_len=sys_len, num_visual=nv,
+                        max_text_len=text, max_decode_steps=2, stride=1, step_ratio_bp=1500, first_prune_layer=0,
+                        tau=4.0)
+    st = torch.cuda.current_stream().cuda_stream
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    f64 = lambda t: t.double().cpu().numpy()
+
+    def attend_kept(q, k, v, ids_sorted):
+        """GPU: causal attention over [S | ids_sorted | I] of one layer's prompt -> (out, scores by original id)."""
+        n = len(ids_sorted)
+        rows = torch.tensor(list(range(sys_len)) + [sys_len + int(i) for i in ids_sorted] +
+                            list(range(sys_len + nv, T)), device="cuda")
+        qs, ks, vs = (t.index_select(1, rows).contiguous() for t in (q, k, v))
+        out = torch.empty_like(qs)
+        probs = torch.zeros(H, max(1, n), device="cuda")
+        scores = torch.full((1, nv), 7.0, device="cuda")
+        ids_dev = torch.tensor(ids_sorted, dtype=torch.int32, device="cuda").reshape(1, -1)
+        B.st3_prefill_attend_kept(qs.data_ptr(), ks.data_ptr(), vs.data_ptr(), out.data_ptr(), probs.data_ptr(),
+                                  scores.data_ptr(), status.data_ptr(), H, H, len(rows), 128, "bf16", sys_len, n,
+                                  ids_dev.data_ptr(), nv, st)
+        ref_out, A = O.causal_attention(f64(qs), f64(ks), f64(vs))
+        bound = 2.0 ** -8 * (np.matmul(A, np.abs(f64(vs))) + np.abs(ref_out)) + 1e-6
+        assert (np.abs(f64(out) - ref_out) - bound).max() <= 0
+        ref_scores = np.full(nv, -1.0)
+        ref_scores[np.asarray(ids_sorted, dtype=np.int64)] = A[:, -1, sys_len:sys_len + n].sum(axis=0)
+        return scores, ref_scores
+
+    ctx = B.Context(cfg)
+    try:
+        scores, ref_scores = attend_kept(Qp, Kp, Vp, list(range(nv)))       # alpha of the layer ahead: all tokens
+        held = set(range(nv))
+        out = torch.empty(1, 1, H, 128, dtype=torch.bfloat16, device="cuda")
+        for l in range(L):
+            got = scores[0].cpu().numpy()
+            mask = ref_scores >= 0
+            assert np.array_equal(got[~mask], ref_scores[~mask])            # tokens not held: exactly -1
+            assert np.allclose(got[mask], ref_scores[mask], rtol=2e-3, atol=1e-7)
+            n_l = B.st3_schedule_count(cfg, l, 0)
+            ctx.prefill_select_scored(Q[l, :, -1].reshape(1, 1, H, 128).contiguous(), K[l].reshape(1, 1, H, T, 128),
+                                      V[l].reshape(1, 1, H, T, 128), [text], scores.reshape(1, 1, nv), out,
+                                      layer_begin=l)
+            ids, cnt, _ = ctx.get_kept(l)
+            kept = ids[0, :int(cnt[0])].cpu().numpy()
+            assert check_kept(ref_scores, np.arange(nv), n_l, kept) in ("exact", "near-tie")
+            assert set(kept.tolist()) <= held and len(kept) == n_l
+            held = set(kept.tolist())
+            # the layer's output for the last prompt token, on the rows it kept (oracle on the GPU's kept set)
+            forced = np.where(np.isin(np.arange(nv), kept), 1.0, 0.0)
+            ref_o, _ = O.prefill_select_scored(f64(Q[l, :, -1]), f64(K[l]), f64(V[l]), sys_len, nv, n_l, forced)
+            rel = np.abs(f64(out[0, 0]) - ref_o) / np.maximum(np.abs(ref_o), 1e-2)
+            assert rel.max() <= 2e-2
+            scores, ref_scores = attend_kept(Q[l], K[l], V[l], sorted(held))  # alpha^l prunes layer l+1
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0 and ctx.status() == 0
+    finally:
+        ctx.close()
+
+
 def test_unsupported_shapes_are_refused():
     x = torch.zeros(1, 8, 64, device="cuda")
     with pytest.raises(B.St3Error) as e:

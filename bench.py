@@ -33,12 +33,14 @@ METRIC = "decode-step attn+trim tokens/s at LLaVA-1.5-7B shape"
 UNIT = "tokens/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic of the attention kernel measured once with ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum over three launches of the llava15_7b workload, see profiles/), as a
-# ratio to the algorithmic bytes of the same launches.  Valid only for the kernel source it was
-# taken on: the hash covers csrc/st3_common.cuh and csrc/st3_attend.cuh.
-ATTEND_TRAFFIC = {"workload": "llava15_7b", "ratio": 1.016,
-                  "kernel_sha256": "b9e81a8572e45e1af4f2282613890dae72ec2472a868d75781ae8e57d5ab47f9"}
+# DRAM traffic of the attention kernel measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum over
+# three launches, see profiles/), as a ratio to the algorithmic bytes of the same launches.  llava15_7b: decode
+# steps 43-45.  llava15_7b_b32: captured on a cut of the workload small enough for the profiler (4 of its 32
+# sequences, decode steps 5-7); a launch's traffic grows in proportion to its sequences (every sequence brings
+# its own rows, nothing is shared), so the ratio carries over to the full batch.  Valid only for the kernel
+# source it was taken on: the hash covers csrc/st3_common.cuh and csrc/st3_attend.cuh.
+ATTEND_TRAFFIC = {"kernel_sha256": "6241ff7b8dda89b239ff1f76d267d3b0ab0a9ccea2642b25bc1ca30e81b08801",
+                  "ratio": {"llava15_7b": 1.015, "llava15_7b_b32": 1.021}}
 
 
 def attend_kernel_sha256():
@@ -51,8 +53,8 @@ def attend_kernel_sha256():
 
 def attend_traffic_ratio(workload_name):
     try:
-        if attend_kernel_sha256() == ATTEND_TRAFFIC["kernel_sha256"] and workload_name == ATTEND_TRAFFIC["workload"]:
-            return ATTEND_TRAFFIC["ratio"]
+        if attend_kernel_sha256() == ATTEND_TRAFFIC["kernel_sha256"]:
+            return ATTEND_TRAFFIC["ratio"].get(workload_name)
     except Exception:
         pass
     return None
@@ -576,7 +578,7 @@ def kernel_roofline(job, steps, world):
     alg = sum(attend_bytes(wl, job.cfg, B, job.text, t) for t in range(0, wl.decode_steps + 1)) * steps
     peak, peak_kind = measured_peak()
     achieved = alg / (attn_ms * 1e-3) / 1e9
-    ratio = attend_traffic_ratio(wl.name) if world == 1 else None
+    ratio = attend_traffic_ratio(wl.name) if world == 1 and not job.cfg.lazy_mask else None
     return {"bound": "hbm", "kernel": "st3_attend_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
             "frac": achieved / peak, "peak_source": f"of {peak_kind}",
             "traffic": None if ratio is None else ratio * alg / max(1, n_attn),
@@ -594,6 +596,26 @@ def add_path_fraction(roofline, job, ms_per_generation):
     roofline["path_achieved"] = pb / (ms_per_generation * 1e-3) / 1e9
     roofline["path_frac"] = roofline["path_achieved"] / roofline["peak"]
     return roofline
+
+
+def per_layer_leg(job, n):
+    """One library call per layer (the calling pattern of a real decoder): tokens/s, GPU time per call, and the
+    host time one st3_decode_step(layer_count=1) call takes (wall clock around a generation's calls, which
+    only enqueue work; the queue is drained before and after)."""
+    wl = job.wl
+    job.generation_per_layer()
+    ms = timed(job.generation_per_layer, n, False)
+    job.ctx.status()
+    calls = wl.num_layers * (wl.decode_steps + 1)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    job.generation_per_layer()
+    host_s = time.perf_counter() - t0
+    torch.cuda.synchronize()
+    job.ctx.status()
+    return {"value": wl.batch * wl.decode_steps * n / (ms * 1e-3), "unit": UNIT, "calls_per_generation": calls,
+            "gpu_us_per_call": ms * 1e3 / (n * calls), "host_us_per_call": host_s * 1e6 / calls,
+            "host_note": "includes the ctypes call overhead of this benchmark's Python loop"}
 
 
 def qk_heredity_line(wl, device, args, name, mask):
@@ -648,6 +670,8 @@ def main():
     ap.add_argument("--workload", default="llava15_7b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--rows-per-chunk", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0, help="run a cut of the workload with this many sequences")
+    ap.add_argument("--decode-steps", type=int, default=0, help="... and this many decode steps (tau unchanged)")
     ap.add_argument("--stage-shared", action="store_true",
                     help="layers between two pruning layers keep the pruning layer's tokens (strided pruning)")
     ap.add_argument("--lazy-mask", type=lambda x: int(x, 0), default=0,
@@ -655,11 +679,14 @@ def main():
     ap.add_argument("--no-extras", action="store_true", help="skip the e2e, unpruned and cpu_baseline legs")
     ap.add_argument("--e2e-only", action="store_true", help="after the timed run, only the end-to-end leg")
     ap.add_argument("--no-others", action="store_true", help="skip the one-generation runs of the other workloads")
-    ap.add_argument("--leg", default="", choices=["", "prefill_attend", "qk_heredity"],
+    ap.add_argument("--leg", default="", choices=["", "prefill_attend", "qk_heredity", "per_layer"],
                     help="run one auxiliary leg alone and print its JSON (for timing or profiling that kernel)")
     ap.add_argument("--instances", type=int, default=2048, help="cap on the (sequence, head) instances of --leg")
     args = ap.parse_args()
     wl = get_workload(args.workload)
+    if args.batch or args.decode_steps:   # a cut of a workload (for profiler captures that must stay small)
+        wl = wl.scaled(name=f"{wl.name}[batch={args.batch or wl.batch},steps={args.decode_steps or wl.decode_steps}]",
+                       batch=args.batch or wl.batch, decode_steps=args.decode_steps or wl.decode_steps)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -718,6 +745,12 @@ def main():
                 qk_heredity_line(wl, device, args, name, mask) for name, mask in (
                     ("stage_shared, no lazy layer", 0), ("layers 29-30 inherit layer 28", (1 << 29) | (1 << 30)),
                     ("layers 4-6 inherit layer 3, layers 8-9 inherit layer 7", sum(1 << l for l in (4, 5, 6, 8, 9))))]}))
+        return
+    if args.leg == "per_layer":
+        if rank == 0:
+            job = Job(wl, device, rows_per_chunk=args.rows_per_chunk)
+            print(json.dumps({"leg": args.leg, "workload": wl.name, **per_layer_leg(job, max(1, args.steps))}))
+            job.ctx.close()
         return
     if dist:
         torch.distributed.init_process_group("nccl", device_id=device)
@@ -798,15 +831,12 @@ def main():
         # prefill-select alone, the one-call-per-layer pattern, and K/V held along a generation
         ms_pre = timed(job.prefill_only, args.steps, False)
         line["prefill_select_ms"] = ms_pre / args.steps
-        job.generation_per_layer()
-        ms_pl = timed(job.generation_per_layer, max(1, args.steps // 2), False)
-        job.ctx.status()
-        line["per_layer_calls"] = {"value": tokens_per_gen * max(1, args.steps // 2) / (ms_pl * 1e-3), "unit": UNIT}
+        line["per_layer_calls"] = per_layer_leg(job, max(1, args.steps // 2))
         line["kv_held"] = job.rows_held_curve()
         line["kept_sets"] = job.kept_set_curve()
         line["prefill_attend"] = prefill_attend_leg(wl, device)
         # the oracle on the host cores, bounded sample
-        ns = 24 if wl.batch == 1 else max(1, 24 // wl.batch)
+        ns = 96 if wl.batch == 1 else max(1, 96 // wl.batch)    # about 10-20 s of host time
         K, V, q0 = job.K.cpu(), job.V.cpu(), job.q0.cpu()
         q, kn, vn = job.q[:ns + 2].cpu(), job.kn[:ns + 2].cpu(), job.vn[:ns + 2].cpu()
         val, secs, threads, s_first, s_last = oracle_sample(wl, job.g, K, V, q0, q, kn, vn, ns, 2)

@@ -76,3 +76,22 @@ def test_argument_validation_without_gpu():
     assert lib.st3_decode_step(None, 1, 0, 1, None, None, None, None, None) == 1
     assert lib.st3_destroy(None) == 1
     assert B.st3_status_string(3) == "call order violated"
+
+
+def test_workspace_grows_by_the_prompt_staging_areas_only_on_request():
+    """host_prefill = 1 adds two slots of one layer's prompt K and V (each rounded up to 256 bytes), nothing else."""
+    a = B.st3_workspace_size(_cfg())
+    b = B.st3_workspace_size(_cfg(host_prefill=1))
+    layer = 1 * 32 * (35 + 576 + 64) * 128 * 2                     # B * H * t0_max * D * bytes
+    assert b - a == 2 * 2 * ((layer + 255) // 256 * 256)
+    # the decode staging (two slots of q | k_new | v_new and of out) is always there: the size depends on L, B, H, D
+    assert B.st3_workspace_size(_cfg(num_layers=16)) < a
+
+
+def test_host_buffer_calls_validate_before_touching_the_gpu():
+    lib = B.load()
+    assert lib.st3_prefill_select_host(None, 0, 1, None, None, None, None, None, None) == 1
+    assert lib.st3_decode_step_host(None, 1, 0, 1, None, None, None, None, None) == 1
+    assert lib.st3_host_sync(None, None) == 1
+    assert lib.st3_prefill_attend_kept(None, None, None, None, None, None, None, 1, 1, 8, 128, 1, 0, 0, None, 8,
+                                       None) == 1

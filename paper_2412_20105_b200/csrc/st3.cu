@@ -218,7 +218,7 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
     ctx->launches++;
   }
   if (select_first) {  // prune by the caller's scores before the layer attends
-    st3_finish_kernel<T, D><<<(unsigned)(2 * p.layer_count * c.batch), kFinishThreads, ctx->finish_smem, st>>>(
+    st3_finish_kernel<T, D, kFinishThreads><<<(unsigned)(2 * p.layer_count * c.batch), kFinishThreads, ctx->finish_smem, st>>>(
         *select_first);
     ctx->launches++;
   }
@@ -261,7 +261,9 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
     // resident as that grid drains and their first instruction waits for all of it.
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(2 * p.layer_count * c.batch));
-    cfg.blockDim = dim3(kFinishThreads);
+    // half-size blocks, two per SM, once the units outnumber the blocks the GPU holds (see st3_finish.cuh)
+    const bool half = 2 * p.layer_count * c.batch > 2 * ctx->num_sms && 2 * ctx->finish_smem <= 200 * 1024;
+    cfg.blockDim = dim3(half ? kFinishThreads / 2 : kFinishThreads);
     cfg.dynamicSmemBytes = (size_t)ctx->finish_smem;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -269,7 +271,9 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = ctx->profiling ? 0 : 1;
-    if (cudaLaunchKernelEx(&cfg, st3_finish_kernel<T, D>, p) != cudaSuccess) return ST3_ERR_CUDA;
+    if ((half ? cudaLaunchKernelEx(&cfg, st3_finish_kernel<T, D, kFinishThreads / 2>, p)
+              : cudaLaunchKernelEx(&cfg, st3_finish_kernel<T, D, kFinishThreads>, p)) != cudaSuccess)
+      return ST3_ERR_CUDA;
   }
   if (e2) cudaEventRecord(e2, st);
   ctx->launches += 2;
@@ -283,7 +287,9 @@ st3_status set_attrs_t(st3_ctx* ctx) {
       cudaFuncSetAttribute(st3_attend_kernel<T, D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            ctx->attend_smem) != cudaSuccess)
     return ST3_ERR_CUDA;
-  if (cudaFuncSetAttribute(st3_finish_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (cudaFuncSetAttribute(st3_finish_kernel<T, D, kFinishThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           ctx->finish_smem) != cudaSuccess ||
+      cudaFuncSetAttribute(st3_finish_kernel<T, D, kFinishThreads / 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            ctx->finish_smem) != cudaSuccess)
     return ST3_ERR_CUDA;
   return ST3_OK;

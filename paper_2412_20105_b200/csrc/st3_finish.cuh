@@ -14,7 +14,6 @@ namespace {
 //               probabilities, radix-selects the rows to keep, pairs holes with kept tail rows and
 //               moves the rows.
 // Both are chains of dependent memory round trips, so every phase issues all its loads first.
-constexpr int kFinishWarps = kFinishThreads / 32;
 constexpr int kHeadBatch = 16;  // logits of one visual row a thread keeps in flight
 
 // (max, 1/sum) of one head's merged softmax from its chunk partials; every lane gets both.
@@ -35,8 +34,11 @@ __device__ __forceinline__ void merge_stats(const float2* ml, long long item0, i
   L = warp_sum(L);
 }
 
-template <typename T, int D>
-__global__ void __launch_bounds__(kFinishThreads) st3_finish_kernel(const StepParams p) {
+// NT threads per block: 1024, or 512 (two blocks per SM) when a launch has more (layer, sequence) units than the GPU
+// can hold blocks: the work of a unit is a chain of memory round trips, and more units in flight end sooner.
+template <typename T, int D, int NT>
+__global__ void __launch_bounds__(NT, 1024 / NT) st3_finish_kernel(const StepParams p) {
+  constexpr int kFinishThreads = NT, kFinishWarps = NT / 32;
   constexpr int ROWB = D * sizeof(T);
   constexpr int VPR = ROWB / 16;  // 16-byte vectors per row
   constexpr int DPL = D / 32;

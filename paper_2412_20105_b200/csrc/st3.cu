@@ -240,7 +240,7 @@ st3_status launch_step_t(st3_ctx* ctx, const StepParams& p, int total_items, cud
     // share.  The kernel reads the step's inputs without waiting for the launch ahead of it, which is only
     // right when those inputs were complete before that launch began - hence off unless the caller says so.
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)(ctx->num_sms * ctx->attend_ctas_per_sm));
+    cfg.gridDim = dim3((unsigned)(p.first_dynamic / kSlots));
     cfg.blockDim = dim3(kAttendThreads);
     cfg.dynamicSmemBytes = (size_t)ctx->attend_smem;
     cfg.stream = st;
@@ -405,7 +405,11 @@ st3_status run_step(st3_ctx* ctx, int step, int layer_begin, int layer_count, co
   const long long work_items = (long long)c.batch * (p.wcvp[p.nwork] + (long long)p.nwork * p.ct);
   if (total_items > L.max_items || work_items * c.num_heads > 0x3fffffffLL) return ST3_ERR_CAPACITY;
   p.total_work = (int)(work_items * c.num_heads);
-  p.first_dynamic = ctx->num_sms * ctx->attend_ctas_per_sm * kSlots;
+  // blocks of the attention grid: as many as fit the GPU, fewer when the launch has fewer items than ring slots
+  {
+    const int full = ctx->num_sms * ctx->attend_ctas_per_sm, need = ceil_div(p.total_work, kSlots);
+    p.first_dynamic = (need < full ? (need > 0 ? need : 1) : full) * kSlots;
+  }
 
   StepParams psel;
   if (ext_scores) {  // parameters of the selection-only launch: all Nv rows held, cut to the schedule

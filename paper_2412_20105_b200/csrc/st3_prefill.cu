@@ -199,7 +199,7 @@ st3_prefill_attend_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
   }
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int qt = blockIdx.x, inst = blockIdx.y;
+  const int qt = (int)gridDim.x - 1 - (int)blockIdx.x, inst = blockIdx.y;   // an instance's longest causal prefixes start first
   const int T = p.T;
   const int row_base = inst * T;  // first row of this instance in the [num_inst * T][128] tensors
   // Query tiles are aligned to the END of the prompt: the ragged tile is the first one, where the causal prefix

@@ -881,6 +881,9 @@ def main():
         line["kv_held"] = job.rows_held_curve()
         line["kept_sets"] = job.kept_set_curve()
         line["prefill_attend"] = prefill_attend_leg(wl, device)
+        if wl.name == "llava15_7b":   # and the longest prompt of the workloads (LLaVA-NeXT shape, 8 sequences x 32 heads)
+            line["prefill_attend_long_prompt"] = prefill_attend_leg(get_workload("llava_next_b8"), device, max_instances=256)
+            torch.cuda.empty_cache()
         # the oracle on the host cores, bounded sample
         ns = 96 if wl.batch == 1 else max(1, 96 // wl.batch)    # about 10-20 s of host time
         K, V, q0 = job.K.cpu(), job.V.cpu(), job.q0.cpu()
